@@ -1,0 +1,193 @@
+/*
+ * gorio.h -- C ABI of the GPU-owned paged graph beam search.
+ *
+ * One B200 runs batched DiskANN-style beam search over a graph index stored as 4 KB
+ * pages.  The GPU owns query evolution, the HBM page cache, page-miss generation,
+ * pending-query state and resume decisions; a thin host proxy thread only services
+ * page reads from the "remote" tier, which is emulated as pinned host memory with an
+ * injected per-request latency (paper: Section 3.1 ownership split, Section 3.2 request
+ * descriptors and per-slot ready table, Section 3.3 persistent scheduler and proxy).
+ *
+ * Conventions
+ *   - Every function returns a gorio_status; nothing throws, aborts or traps.
+ *   - "device" pointers are CUDA device memory of the index's device; "host" pointers
+ *     are ordinary host memory.  No torch or C++ types cross this boundary.
+ *   - The library needs its CUDA kernels: there is no CPU fallback of any kind.
+ *   - A gorio_index is not thread safe; use one caller thread per index.
+ */
+#ifndef GORIO_H
+#define GORIO_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gorio_index gorio_index; /* opaque; created by gorio_index_open, freed by gorio_index_close */
+
+typedef enum {
+  GORIO_OK = 0,
+  GORIO_ERR_INVALID_ARG = 1,   /* a precondition listed at the call does not hold */
+  GORIO_ERR_CUDA = 2,          /* a CUDA runtime call failed (see gorio_last_error) */
+  GORIO_ERR_NOMEM = 3,         /* device or host allocation failed */
+  GORIO_ERR_STATE = 4,         /* call order: search before cache_config, ... */
+  GORIO_ERR_TIMEOUT = 5,       /* a bounded device or host wait expired; all kernels have exited */
+  GORIO_ERR_CAPACITY = 6,      /* per-query visited/page set or iteration limit exhausted */
+  GORIO_ERR_INDEX_CORRUPT = 7, /* neighbour id >= n_nodes or degree > max_degree met in a page */
+  GORIO_ERR_INTERNAL = 8       /* a self-check of the cache/scheduler state machine failed */
+} gorio_status;
+
+enum { GORIO_DTYPE_U8 = 0, GORIO_DTYPE_F32 = 1 };
+enum { GORIO_FLAG_PAGES_ALREADY_PINNED = 1u }; /* host_pages is already page-locked and mapped */
+
+/*
+ * Index description (Section 5.1: "on-disk graph index"; the layout below is this
+ * library's page-store format).
+ *   Node i lives in page i / nodes_per_page at byte (i % nodes_per_page) * node_bytes,
+ *   node_bytes = dim*elem_size + 4 + 4*max_degree.  A node is: vector[dim] (u8 or LE f32),
+ *   degree (u32 LE), max_degree neighbour ids (u32 LE, unused entries 0xFFFFFFFF).
+ *   host_pages: n_pages * 4096 bytes of HOST memory, owned by the caller and borrowed
+ *   until gorio_index_close.  It is the emulated remote tier; the library page-locks it
+ *   (cudaHostRegister) unless GORIO_FLAG_PAGES_ALREADY_PINNED is set.
+ *   PQ navigation (optional): pq_m > 0 enables it; pq_centroids_dev is u8
+ *   [pq_m][256][dim/pq_m] and pq_codes_dev is u8 [n_nodes][pq_m], both DEVICE memory
+ *   borrowed until close.  Requires dtype u8, dim % pq_m == 0, (dim/pq_m) % 4 == 0.
+ * Preconditions: page_bytes == 4096, dim % 4 == 0, nodes_per_page*node_bytes <= 4096,
+ *   n_nodes < 2^31, entry_id < n_nodes, max_degree >= 1.
+ */
+typedef struct {
+  uint64_t n_nodes;
+  uint32_t dim;
+  uint32_t dtype;
+  uint32_t max_degree;
+  uint32_t nodes_per_page;
+  uint32_t page_bytes;
+  uint32_t entry_id; /* medoid entry node */
+  const void *host_pages;
+  uint32_t pq_m;
+  uint32_t flags;
+  const uint8_t *pq_centroids_dev;
+  const uint8_t *pq_codes_dev;
+} gorio_index_desc;
+
+/*
+ * Page cache + remote tier configuration (Section 3.2: GPU page-cache slots with one
+ * ready entry each; Section 3.3: the proxy "batches submissions and completions,
+ * controls outstanding remote I/O").
+ *   capacity_pages   HBM cache size in 4 KB slots.  The cache is a 16-way set-associative
+ *                    lock-free hash with a clock hand per set; capacity is rounded down
+ *                    to a multiple of 16, except that capacity >= n_pages makes every
+ *                    page resident-capable.  Must be >= 16.
+ *   remote_latency_ns  a request's completion is published no earlier than this long
+ *                    after the proxy admitted it.
+ *   max_outstanding  most requests admitted and not yet published (>= 1).
+ *   preload          1: fill the cache with pages 0..capacity-1 now (whole index when
+ *                    capacity >= n_pages); 0: start cold.
+ *   timeout_ms       bound on one gorio_search call (device and host waits); 0 = 60000.
+ *   copy_mode        0: the proxy enqueues batched gather-copy kernels on its own streams;
+ *                    1: the proxy issues one cudaMemcpyAsync per page (DMA engine).
+ *   fill_batch       pages per proxy copy batch (1..128), 0 = default.
+ * Calling it again re-creates an empty (or preloaded) cache.
+ */
+typedef struct {
+  uint64_t capacity_pages;
+  uint32_t remote_latency_ns;
+  uint32_t max_outstanding;
+  uint32_t preload;
+  uint32_t timeout_ms;
+  uint32_t copy_mode;
+  uint32_t fill_batch;
+} gorio_cache_cfg;
+
+/*
+ * Scheduler tuning; all zero = defaults.
+ *   max_inflight     query slots resident at once (pending/running queries); default 16384.
+ *   visited_capacity per-query exact visited-set entries (power of two), default 32768;
+ *                    a query that scores more nodes fails with GORIO_ERR_CAPACITY.
+ *   warps_per_block / blocks_per_sm  launch geometry of the persistent kernel.
+ */
+typedef struct {
+  uint32_t max_inflight;
+  uint32_t visited_capacity;
+  uint32_t warps_per_block;
+  uint32_t blocks_per_sm;
+} gorio_tuning;
+
+/*
+ * Counters since the last gorio_stats_reset.
+ *   pages_hit      page lookups satisfied from a resident slot
+ *   pages_missed   (query, node) waits registered on a page in flight (owner or joiner)
+ *   pages_fetched  request descriptors the proxy serviced (4 KB each)
+ *   dedupe_joins   waits that joined another query's or lane's outstanding request
+ *   evictions, retries (lookups deferred because the set had no evictable slot or a
+ *   validation failed), max_outstanding_seen (proxy), queries_done,
+ *   n_eval / n_expand / sum_degree: totals of the per-query search counters (used for
+ *   the algorithmic byte count), search_ns: wall time of the blocking search calls.
+ * Hit/miss/fetch counts depend on timing; they obey invariants, not fixed values.
+ */
+typedef struct {
+  uint64_t pages_hit, pages_missed, pages_fetched;
+  uint64_t dedupe_joins, evictions, retries, max_outstanding_seen, queries_done;
+  uint64_t n_eval, n_expand, sum_degree, n_iter;
+  uint64_t resumes, search_ns, proxy_batches, reserved0;
+} gorio_stats_t;
+
+/* Open an index on CUDA device `cuda_device`.  *out is set only on GORIO_OK. */
+int gorio_index_open(const gorio_index_desc *desc, int cuda_device, gorio_index **out);
+
+/* (Re)create the page cache and arm the remote-tier emulation.  Blocking. */
+int gorio_cache_config(gorio_index *ix, const gorio_cache_cfg *cfg);
+
+/* Optional; takes effect at the next gorio_search. */
+int gorio_set_tuning(gorio_index *ix, const gorio_tuning *t);
+
+/*
+ * Batched beam search (Section 2.2: expand nodes, evaluate distances, update the
+ * candidate list, discover the next pages; Section 3.3: queries that miss are parked
+ * and resumed by the GPU scheduler).  For every query: start at entry_id; repeatedly
+ * take the first W unexpanded entries of the L-entry list ordered by (distance, id),
+ * read their adjacency from their pages, score every not-yet-visited neighbour (exact
+ * navigation: from the neighbour's own page; PQ navigation: from resident codes) and keep
+ * the L best; stop when no unexpanded entry remains.  Output the best K by (distance, id)
+ * (PQ navigation: best K expanded nodes by exact distance).
+ *
+ *   queries_dev   DEVICE [nq][dim], index dtype, row major.
+ *   out_ids_dev   DEVICE [nq][K] u32; out_dists_dev DEVICE [nq][K] (u32 for u8 data, f32
+ *                 for f32 data).  Missing results are 0xFFFFFFFF / 0xFFFFFFFF or +inf.
+ *   out_pages_distinct_dev  DEVICE [nq] u32 or NULL: distinct pages each query touched.
+ *   out_counters_dev        DEVICE [nq][5] u32 or NULL: pages_distinct, iterations,
+ *                 expansions, evaluations, sum of expanded degrees.
+ *   cuda_stream   cudaStream_t (or NULL for the default stream) used for the launches.
+ * Preconditions: 1 <= K <= L <= 256, 1 <= W <= 16, W*max_degree <= 1024, nq >= 1.
+ * Blocking: returns after all queries finished (results visible on the device) or with an
+ * error status after every kernel and proxy action of this call has ended.
+ */
+int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t K, uint32_t L,
+                 uint32_t W, uint32_t *out_ids_dev, void *out_dists_dev,
+                 uint32_t *out_pages_distinct_dev, uint32_t *out_counters_dev, void *cuda_stream);
+
+/*
+ * The same search with HOST buffers: queries are copied host->device, results
+ * device->host, inside the call (the end-to-end path).  out_pages_distinct_host and
+ * out_counters_host may be NULL.
+ */
+int gorio_search_host(gorio_index *ix, const void *queries_host, uint32_t nq, uint32_t K,
+                      uint32_t L, uint32_t W, uint32_t *out_ids_host, void *out_dists_host,
+                      uint32_t *out_pages_distinct_host, uint32_t *out_counters_host);
+
+int gorio_stats(gorio_index *ix, gorio_stats_t *out);
+int gorio_stats_reset(gorio_index *ix);
+
+/* Stops the proxy thread, frees every device and host resource of the index. */
+int gorio_index_close(gorio_index *ix);
+
+/* Static strings; never NULL. */
+const char *gorio_status_str(int status);
+/* Human-readable detail of the last non-OK status on this index (valid until the next call). */
+const char *gorio_last_error(gorio_index *ix);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GORIO_H */

@@ -1,0 +1,617 @@
+// Host side of the C ABI declared in include/gorio.h: resource management, the blocking
+// search call, and the CPU proxy thread that services page requests from the emulated
+// remote tier (paper Section 3.3: the proxy "batches submissions and completions, controls
+// outstanding remote I/O, and publishes ready state", and never looks at search state).
+#include <atomic>
+#include <chrono>
+#include <condition_variable>
+#include <cstdio>
+#include <cstring>
+#include <deque>
+#include <mutex>
+#include <new>
+#include <string>
+#include <thread>
+#include <vector>
+
+#include "../../include/gorio.h"
+#include "gorio_internal.h"
+
+using namespace gorio;
+
+namespace {
+
+constexpr int kMaxFillStreams = 4;
+typedef std::chrono::steady_clock Clock;
+
+inline u32 next_pow2(u64 v) { u32 p = 1; while (p < v) p <<= 1; return p; }
+inline u32 ilog2(u32 v) { u32 s = 0; while ((1u << s) < v) ++s; return s; }
+
+enum ProxyState : int { PX_IDLE = 0, PX_RUN = 1, PX_EXIT = 2 };
+
+}  // namespace
+
+struct gorio_index {
+  gorio_index_desc desc{};
+  int dev = 0;
+  int n_sms = 0;
+  u32 n_pages = 0, node_bytes = 0, vec_bytes = 0;
+  bool registered_pages = false;
+  const u8 *pages_dev = nullptr;   // device view of the host page store
+
+  // cache
+  gorio_cache_cfg cfg{};
+  bool cache_ready = false, cache_dirty = false;
+  u32 n_sets = 0, n_slots = 0, preloaded = 0;
+  u8 *slot_data = nullptr;
+  u64 *tag = nullptr, *wl = nullptr;
+  u32 *hand = nullptr;
+  // host-mapped communication areas
+  u64 *ring_h = nullptr; u64 *ring_d = nullptr; u32 ring_cap = 0;
+  u32 *comp_h = nullptr; u32 *comp_d = nullptr;
+  u32 *hctl_h = nullptr; u32 *hctl_d = nullptr;     // [0] completion tail, [1] abort, [8..] copied flags
+  u32 *fill_counters = nullptr;                     // device, one per fill stream
+  u64 *arr_buf = nullptr;
+
+  // query state
+  gorio_tuning tune{};
+  u32 qs_slots = 0, qs_L = 0, qs_W = 0, qs_WR = 0, qs_K = 0, qs_seen = 0, qs_pset = 0;
+  void *qs_block = nullptr;
+  Ctx ctx{};
+  Ctl *ctl = nullptr;
+  u64 *run_buf = nullptr, *retry_buf = nullptr; u32 runq_cap = 0;
+
+  // host-buffer search staging
+  void *st_q = nullptr; size_t st_q_bytes = 0;
+  void *st_out = nullptr; size_t st_out_bytes = 0;
+
+  // proxy
+  std::thread proxy;
+  std::mutex mu;
+  std::condition_variable cv;
+  std::atomic<int> px_state{PX_IDLE};
+  std::atomic<int> px_stop{0};
+  std::atomic<int> px_active{0};
+  std::atomic<int> px_error{0};
+  cudaStream_t fill_streams[kMaxFillStreams] = {};
+  cudaStream_t own_stream = nullptr;
+  cudaEvent_t done_ev = nullptr;
+
+  // statistics
+  u64 host_fetched = 0, host_max_out = 0, host_batches = 0, host_search_ns = 0;
+  u32 px_dbg[8] = {};   // proxy progress at the end of its last service loop
+  std::string err;
+};
+
+namespace {
+
+int fail(gorio_index *ix, int status, const std::string &msg) {
+  if (ix) ix->err = msg;
+  return status;
+}
+int cuda_fail(gorio_index *ix, cudaError_t e, const char *what) {
+  return fail(ix, e == cudaErrorMemoryAllocation ? GORIO_ERR_NOMEM : GORIO_ERR_CUDA,
+              std::string(what) + ": " + cudaGetErrorString(e));
+}
+#define CK(call)                                                         \
+  do {                                                                   \
+    cudaError_t e__ = (call);                                            \
+    if (e__ != cudaSuccess) return cuda_fail(ix, e__, #call);            \
+  } while (0)
+
+template <typename T>
+cudaError_t host_mapped(T **h, T **d, size_t count) {
+  void *p = nullptr;
+  cudaError_t e = cudaHostAlloc(&p, count * sizeof(T), cudaHostAllocMapped | cudaHostAllocPortable);
+  if (e != cudaSuccess) return e;
+  std::memset(p, 0, count * sizeof(T));
+  *h = (T *)p;
+  void *dp = nullptr;
+  e = cudaHostGetDevicePointer(&dp, p, 0);
+  *d = (T *)dp;
+  return e;
+}
+
+void free_cache(gorio_index *ix) {
+  cudaFree(ix->slot_data); cudaFree(ix->tag); cudaFree(ix->wl); cudaFree(ix->hand);
+  cudaFree(ix->arr_buf); cudaFree(ix->fill_counters);
+  if (ix->ring_h) cudaFreeHost(ix->ring_h);
+  if (ix->comp_h) cudaFreeHost(ix->comp_h);
+  ix->slot_data = nullptr; ix->tag = ix->wl = nullptr; ix->hand = nullptr; ix->arr_buf = nullptr;
+  ix->fill_counters = nullptr; ix->ring_h = ix->ring_d = nullptr; ix->comp_h = ix->comp_d = nullptr;
+  ix->cache_ready = false;
+}
+
+void free_qstate(gorio_index *ix) {
+  cudaFree(ix->qs_block); cudaFree(ix->run_buf); cudaFree(ix->retry_buf);
+  ix->qs_block = nullptr; ix->run_buf = ix->retry_buf = nullptr; ix->qs_slots = 0;
+}
+
+// ---------------------------------------------------------------------------------------
+// the proxy: consumes request descriptors in order, bounds the number in service, moves
+// page bytes from pinned host memory into cache slots, and publishes completions no
+// earlier than admission + latency.
+// ---------------------------------------------------------------------------------------
+__global__ void notify_kernel(u32 *host_copied, u32 seq) {
+  asm volatile("st.relaxed.sys.global.u32 [%0], %1;" ::"l"(host_copied), "r"(seq) : "memory");
+}
+
+struct InService { u32 slot; u32 stream; u32 seq; Clock::time_point admitted; };
+
+void proxy_service(gorio_index *ix) {
+  const u32 ring_mask = ix->ring_cap - 1, ring_shift = ilog2(ix->ring_cap);
+  const u32 max_out = ix->cfg.max_outstanding;
+  const u32 batch_max = ix->cfg.fill_batch;
+  const auto latency = std::chrono::nanoseconds(ix->cfg.remote_latency_ns);
+  const int n_streams = kMaxFillStreams;
+  volatile u64 *ring = ix->ring_h;
+  volatile u32 *copied = ix->hctl_h + 8;
+  u32 tail = 0, ct = 0, outstanding = 0;
+  u32 stream_seq[kMaxFillStreams] = {0, 0, 0, 0};
+  int k = 0;
+  std::deque<InService> inflight;
+  FillBatch batch;
+  u64 fetched = 0, max_seen = 0, batches = 0;
+
+  while (!ix->px_stop.load(std::memory_order_acquire)) {
+    // 1. admit descriptors while the in-service window has room
+    batch.n = 0;
+    const Clock::time_point now0 = Clock::now();
+    while (outstanding < max_out && batch.n < batch_max) {
+      const u64 e = ring[tail & ring_mask];
+      const u32 lap = ((tail >> ring_shift) % 255u) + 1u;
+      if ((u32)(e & 0xFFu) != lap) break;
+      std::atomic_thread_fence(std::memory_order_acquire);
+      batch.page[batch.n] = (u32)(e >> 32);
+      batch.slot[batch.n] = (u32)(e >> 8) & 0xFFFFFFu;
+      if (batch.page[batch.n] >= ix->n_pages || batch.slot[batch.n] >= ix->n_slots) {
+        ix->px_error.store(1);   // a descriptor the GPU could not have produced
+        return;
+      }
+      ++batch.n; ++tail; ++outstanding;
+    }
+    if (batch.n) {
+      const u32 seq = ++stream_seq[k];
+      batch.seq = seq;
+      cudaError_t e = cudaSuccess;
+      if (ix->cfg.copy_mode == 0) {
+        e = launch_fill(batch, ix->pages_dev, ix->slot_data, ix->fill_counters + k,
+                        ix->hctl_d + 8 + k, ix->fill_streams[k]);
+      } else {
+        for (u32 i = 0; i < batch.n && e == cudaSuccess; ++i)
+          e = cudaMemcpyAsync(ix->slot_data + (size_t)batch.slot[i] * kPageBytes,
+                              (const u8 *)ix->desc.host_pages + (size_t)batch.page[i] * kPageBytes,
+                              kPageBytes, cudaMemcpyHostToDevice, ix->fill_streams[k]);
+        if (e == cudaSuccess) {
+          notify_kernel<<<1, 1, 0, ix->fill_streams[k]>>>(ix->hctl_d + 8 + k, seq);
+          e = cudaGetLastError();
+        }
+      }
+      if (e != cudaSuccess) { ix->px_error.store(2); return; }
+      for (u32 i = 0; i < batch.n; ++i) inflight.push_back({batch.slot[i], (u32)k, seq, now0});
+      k = (k + 1) % n_streams;
+      ++batches;
+      if (outstanding > max_seen) max_seen = outstanding;
+    }
+    // 2. publish completions in admission order: copy landed and latency elapsed
+    if (!inflight.empty()) {
+      const Clock::time_point now = Clock::now();
+      u32 published = 0;
+      while (!inflight.empty()) {
+        const InService &r = inflight.front();
+        if (now - r.admitted < latency) break;
+        if ((int)(copied[r.stream] - r.seq) < 0) break;
+        ix->comp_h[ct & ring_mask] = r.slot;
+        ++ct; ++published;
+        inflight.pop_front();
+      }
+      if (published) {
+        std::atomic_thread_fence(std::memory_order_release);
+        ((volatile u32 *)ix->hctl_h)[0] = ct;
+        outstanding -= published;
+        fetched += published;
+      }
+    }
+  }
+  ix->px_dbg[0] = tail; ix->px_dbg[1] = ct; ix->px_dbg[2] = outstanding; ix->px_dbg[3] = (u32)inflight.size();
+  if (!inflight.empty()) {
+    ix->px_dbg[4] = inflight.front().stream; ix->px_dbg[5] = inflight.front().seq;
+    ix->px_dbg[6] = copied[inflight.front().stream];
+  }
+  ix->host_fetched += fetched;
+  ix->host_batches += batches;
+  if (max_seen > ix->host_max_out) ix->host_max_out = max_seen;
+}
+
+void proxy_main(gorio_index *ix) {
+  cudaSetDevice(ix->dev);
+  for (;;) {
+    {
+      std::unique_lock<std::mutex> lk(ix->mu);
+      ix->cv.wait(lk, [&] { return ix->px_state.load() != PX_IDLE; });
+    }
+    if (ix->px_state.load() == PX_EXIT) return;
+    ix->px_active.store(1, std::memory_order_release);
+    proxy_service(ix);
+    {
+      std::lock_guard<std::mutex> lk(ix->mu);
+      if (ix->px_state.load() != PX_EXIT) ix->px_state.store(PX_IDLE);
+      ix->px_active.store(0, std::memory_order_release);
+    }
+    ix->cv.notify_all();
+  }
+}
+
+void proxy_start(gorio_index *ix) {
+  ix->px_stop.store(0);
+  ix->px_error.store(0);
+  {
+    std::lock_guard<std::mutex> lk(ix->mu);
+    ix->px_state.store(PX_RUN);
+  }
+  ix->cv.notify_all();
+}
+
+void proxy_stop(gorio_index *ix) {
+  ix->px_stop.store(1, std::memory_order_release);
+  std::unique_lock<std::mutex> lk(ix->mu);
+  ix->cv.wait(lk, [&] { return ix->px_state.load() == PX_IDLE || ix->px_state.load() == PX_EXIT; });
+}
+
+// ---------------------------------------------------------------------------------------
+int setup_cache(gorio_index *ix) {
+  const gorio_cache_cfg &cfg = ix->cfg;
+  free_cache(ix);
+  const u64 cap = cfg.capacity_pages;
+  if (cap >= ix->n_pages) ix->n_sets = (ix->n_pages + kWays - 1) / kWays;
+  else ix->n_sets = (u32)(cap / kWays);
+  ix->n_slots = ix->n_sets * kWays;
+  ix->ring_cap = next_pow2(2ull * ix->n_slots < 1024 ? 1024 : 2ull * ix->n_slots);
+  CK(cudaMalloc(&ix->slot_data, (size_t)ix->n_slots * kPageBytes));
+  CK(cudaMalloc(&ix->tag, (size_t)ix->n_slots * 8));
+  CK(cudaMalloc(&ix->wl, (size_t)ix->n_slots * 8));
+  CK(cudaMalloc(&ix->hand, (size_t)ix->n_sets * 4));
+  CK(cudaMalloc(&ix->arr_buf, (size_t)ix->ring_cap * 8));
+  CK(cudaMalloc(&ix->fill_counters, kMaxFillStreams * 4));
+  CK(cudaMemset(ix->fill_counters, 0, kMaxFillStreams * 4));
+  CK(host_mapped(&ix->ring_h, &ix->ring_d, ix->ring_cap));
+  CK(host_mapped(&ix->comp_h, &ix->comp_d, ix->ring_cap));
+  // Warm the whole proxy copy path (kernel code, launch path of every copy stream) before a
+  // persistent kernel can depend on it: copy page 0 into slot 0 once per stream.
+  {
+    cudaFuncAttributes fa;
+    CK(cudaFuncGetAttributes(&fa, notify_kernel));
+    FillBatch wb{};
+    wb.n = 1; wb.seq = 0; wb.page[0] = 0; wb.slot[0] = 0;
+    for (int i = 0; i < kMaxFillStreams; ++i) {
+      CK(launch_fill(wb, ix->pages_dev, ix->slot_data, ix->fill_counters + i, ix->hctl_d + 8 + i, ix->fill_streams[i]));
+      notify_kernel<<<1, 1, 0, ix->fill_streams[i]>>>(ix->hctl_d + 8 + i, 0);
+      CK(cudaGetLastError());
+      CK(cudaStreamSynchronize(ix->fill_streams[i]));
+    }
+  }
+  ix->preloaded = 0;
+  if (cfg.preload) {
+    ix->preloaded = cap >= ix->n_pages ? ix->n_pages : ix->n_slots;
+    CK(cudaMemcpy(ix->slot_data, ix->desc.host_pages, (size_t)ix->preloaded * kPageBytes, cudaMemcpyHostToDevice));
+  }
+  Ctx c{};
+  c.tag = ix->tag; c.wl = ix->wl; c.hand = ix->hand; c.n_sets = ix->n_sets; c.n_slots = ix->n_slots;
+  CK(launch_cache_reset(c, ix->preloaded, ix->own_stream));
+  CK(cudaStreamSynchronize(ix->own_stream));
+  ix->cache_ready = true;
+  ix->cache_dirty = false;
+  return GORIO_OK;
+}
+
+int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W) {
+  const u32 R = ix->desc.max_degree, WR = W * R;
+  const u32 max_inflight = ix->tune.max_inflight ? ix->tune.max_inflight : 16384u;
+  const u32 slots = nq < max_inflight ? nq : max_inflight;
+  const u32 seen_cap = ix->tune.visited_capacity ? ix->tune.visited_capacity : 32768u;
+  const u32 pset_cap = ix->desc.pq_m ? 4096u : seen_cap;
+  if (ix->qs_block && ix->qs_slots >= slots && ix->qs_L == L && ix->qs_W == W && ix->qs_K == K &&
+      ix->qs_seen == seen_cap && ix->qs_pset == pset_cap) {
+    ix->ctx.n_qslots = slots;
+    return GORIO_OK;
+  }
+  free_qstate(ix);
+  auto al = [](size_t v) { return (v + 255) & ~(size_t)255; };
+  size_t off = 0;
+  const size_t o_hdr = off;  off += al((size_t)slots * sizeof(QHdr));
+  const size_t o_list = off; off += al((size_t)slots * L * 8);
+  const size_t o_cand = off; off += al((size_t)slots * WR * 8);
+  const size_t o_items = off; off += al((size_t)slots * WR * 4);
+  const size_t o_wrec = off; off += al((size_t)slots * WR * 4);
+  const size_t o_adj = off;  off += al((size_t)slots * WR * 4);
+  const size_t o_adeg = off; off += al((size_t)slots * W * 4);
+  const size_t o_todo = off; off += al((size_t)slots * WR * 2);
+  const size_t o_pool = off; off += al((size_t)slots * (K + W) * 8);
+  const size_t o_seen = off; off += al((size_t)slots * seen_cap * 4);
+  const size_t o_pset = off; off += al((size_t)slots * pset_cap * 4);
+  CK(cudaMalloc(&ix->qs_block, off));
+  ix->runq_cap = next_pow2(2ull * slots < 64 ? 64 : 2ull * slots);
+  CK(cudaMalloc(&ix->run_buf, (size_t)ix->runq_cap * 8));
+  CK(cudaMalloc(&ix->retry_buf, (size_t)ix->runq_cap * 8));
+  u8 *b = (u8 *)ix->qs_block;
+  Ctx &c = ix->ctx;
+  c.hdr = (QHdr *)(b + o_hdr); c.list = (u64 *)(b + o_list); c.cand = (u64 *)(b + o_cand);
+  c.items = (u32 *)(b + o_items); c.wrec = (u32 *)(b + o_wrec); c.adj = (u32 *)(b + o_adj);
+  c.adjdeg = (u32 *)(b + o_adeg); c.todo = (u16 *)(b + o_todo); c.pool = (u64 *)(b + o_pool);
+  c.seen = (u32 *)(b + o_seen); c.pset = (u32 *)(b + o_pset);
+  c.seen_cap = seen_cap; c.pset_cap = pset_cap; c.n_qslots = slots;
+  ix->qs_slots = slots; ix->qs_L = L; ix->qs_W = W; ix->qs_WR = WR; ix->qs_K = K;
+  ix->qs_seen = seen_cap; ix->qs_pset = pset_cap;
+  return GORIO_OK;
+}
+
+const char *kDeviceErr[] = {"", "", "", "", "", "device wait expired", "per-query capacity exhausted",
+                            "corrupt index page", "internal state-machine check failed"};
+
+}  // namespace
+
+// =========================================================================================
+extern "C" {
+
+const char *gorio_status_str(int s) {
+  switch (s) {
+    case GORIO_OK: return "ok";
+    case GORIO_ERR_INVALID_ARG: return "invalid argument";
+    case GORIO_ERR_CUDA: return "CUDA error";
+    case GORIO_ERR_NOMEM: return "out of memory";
+    case GORIO_ERR_STATE: return "call out of order";
+    case GORIO_ERR_TIMEOUT: return "timeout";
+    case GORIO_ERR_CAPACITY: return "capacity exhausted";
+    case GORIO_ERR_INDEX_CORRUPT: return "corrupt index";
+    case GORIO_ERR_INTERNAL: return "internal error";
+    default: return "unknown status";
+  }
+}
+
+const char *gorio_last_error(gorio_index *ix) { return ix ? ix->err.c_str() : ""; }
+
+int gorio_index_open(const gorio_index_desc *d, int cuda_device, gorio_index **out) {
+  if (!d || !out) return GORIO_ERR_INVALID_ARG;
+  const u32 esz = d->dtype == GORIO_DTYPE_U8 ? 1u : 4u;
+  const u64 nb = (u64)d->dim * esz + 4 + 4ull * d->max_degree;
+  if (d->dtype > GORIO_DTYPE_F32 || d->page_bytes != kPageBytes || d->dim == 0 || d->dim % 4 != 0 ||
+      d->max_degree == 0 || d->nodes_per_page == 0 || nb * d->nodes_per_page > kPageBytes ||
+      d->n_nodes == 0 || d->n_nodes >= (1ull << 31) || d->entry_id >= d->n_nodes || !d->host_pages)
+    return GORIO_ERR_INVALID_ARG;
+  if (d->pq_m) {
+    if (d->dtype != GORIO_DTYPE_U8 || d->dim % d->pq_m != 0 || (d->dim / d->pq_m) % 4 != 0 ||
+        d->pq_m > 64 || !d->pq_centroids_dev || !d->pq_codes_dev)
+      return GORIO_ERR_INVALID_ARG;
+  }
+  gorio_index *ix = new (std::nothrow) gorio_index();
+  if (!ix) return GORIO_ERR_NOMEM;
+  ix->desc = *d;
+  ix->dev = cuda_device;
+  ix->node_bytes = (u32)nb;
+  ix->vec_bytes = d->dim * esz;
+  ix->n_pages = (u32)((d->n_nodes + d->nodes_per_page - 1) / d->nodes_per_page);
+  auto bail = [&](int st) { gorio_index_close(ix); return st; };
+  cudaError_t e = cudaSetDevice(cuda_device);
+  if (e != cudaSuccess) return bail(GORIO_ERR_CUDA);
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, cuda_device) != cudaSuccess) return bail(GORIO_ERR_CUDA);
+  ix->n_sms = prop.multiProcessorCount;
+  const size_t bytes = (size_t)ix->n_pages * kPageBytes;
+  if (!(d->flags & GORIO_FLAG_PAGES_ALREADY_PINNED)) {
+    e = cudaHostRegister((void *)d->host_pages, bytes, cudaHostRegisterMapped | cudaHostRegisterPortable);
+    if (e != cudaSuccess) { cudaGetLastError(); return bail(GORIO_ERR_CUDA); }
+    ix->registered_pages = true;
+  }
+  void *dp = nullptr;
+  if (cudaHostGetDevicePointer(&dp, (void *)d->host_pages, 0) != cudaSuccess) return bail(GORIO_ERR_CUDA);
+  ix->pages_dev = (const u8 *)dp;
+  if (preload_kernels() != cudaSuccess) return bail(GORIO_ERR_CUDA);
+  if (host_mapped(&ix->hctl_h, &ix->hctl_d, 64) != cudaSuccess) return bail(GORIO_ERR_CUDA);
+  if (cudaMalloc(&ix->ctl, sizeof(Ctl)) != cudaSuccess) return bail(GORIO_ERR_NOMEM);
+  cudaMemset(ix->ctl, 0, sizeof(Ctl));
+  int lo = 0, hi = 0;
+  cudaDeviceGetStreamPriorityRange(&lo, &hi);
+  for (int i = 0; i < kMaxFillStreams; ++i)
+    if (cudaStreamCreateWithPriority(&ix->fill_streams[i], cudaStreamNonBlocking, hi) != cudaSuccess)
+      return bail(GORIO_ERR_CUDA);
+  if (cudaStreamCreateWithFlags(&ix->own_stream, cudaStreamNonBlocking) != cudaSuccess) return bail(GORIO_ERR_CUDA);
+  if (cudaEventCreateWithFlags(&ix->done_ev, cudaEventDisableTiming) != cudaSuccess) return bail(GORIO_ERR_CUDA);
+  ix->proxy = std::thread(proxy_main, ix);
+  *out = ix;
+  return GORIO_OK;
+}
+
+int gorio_index_close(gorio_index *ix) {
+  if (!ix) return GORIO_ERR_INVALID_ARG;
+  cudaSetDevice(ix->dev);
+  if (ix->proxy.joinable()) {
+    ix->px_stop.store(1);
+    {
+      std::lock_guard<std::mutex> lk(ix->mu);
+      ix->px_state.store(PX_EXIT);
+    }
+    ix->cv.notify_all();
+    ix->proxy.join();
+  }
+  cudaDeviceSynchronize();
+  free_cache(ix);
+  free_qstate(ix);
+  cudaFree(ix->ctl);
+  cudaFree(ix->st_q); cudaFree(ix->st_out);
+  if (ix->hctl_h) cudaFreeHost(ix->hctl_h);
+  for (int i = 0; i < kMaxFillStreams; ++i) if (ix->fill_streams[i]) cudaStreamDestroy(ix->fill_streams[i]);
+  if (ix->own_stream) cudaStreamDestroy(ix->own_stream);
+  if (ix->done_ev) cudaEventDestroy(ix->done_ev);
+  if (ix->registered_pages) cudaHostUnregister((void *)ix->desc.host_pages);
+  delete ix;
+  return GORIO_OK;
+}
+
+int gorio_cache_config(gorio_index *ix, const gorio_cache_cfg *cfg) {
+  if (!ix || !cfg) return GORIO_ERR_INVALID_ARG;
+  if (cfg->capacity_pages < kWays || cfg->max_outstanding < 1 || cfg->copy_mode > 1 ||
+      cfg->fill_batch > kMaxFillBatch)
+    return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: capacity >= 16, max_outstanding >= 1, copy_mode 0|1, fill_batch <= 128");
+  u64 cap = cfg->capacity_pages < ix->n_pages ? cfg->capacity_pages : ix->n_pages;
+  if (cap / kWays * kWays >= (1ull << 24)) return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: at most 2^24 slots");
+  CK(cudaSetDevice(ix->dev));
+  ix->cfg = *cfg;
+  if (ix->cfg.timeout_ms == 0) ix->cfg.timeout_ms = 60000;
+  if (ix->cfg.fill_batch == 0) ix->cfg.fill_batch = 64;
+  return setup_cache(ix);
+}
+
+int gorio_set_tuning(gorio_index *ix, const gorio_tuning *t) {
+  if (!ix || !t) return GORIO_ERR_INVALID_ARG;
+  if (t->visited_capacity && ((t->visited_capacity & (t->visited_capacity - 1)) || t->visited_capacity < 64))
+    return fail(ix, GORIO_ERR_INVALID_ARG, "visited_capacity must be a power of two >= 64");
+  if (t->warps_per_block > 32) return fail(ix, GORIO_ERR_INVALID_ARG, "warps_per_block <= 32");
+  ix->tune = *t;
+  return GORIO_OK;
+}
+
+int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t K, uint32_t L, uint32_t W,
+                 uint32_t *out_ids_dev, void *out_dists_dev, uint32_t *out_pages_distinct_dev,
+                 uint32_t *out_counters_dev, void *cuda_stream) {
+  if (!ix) return GORIO_ERR_INVALID_ARG;
+  if (!queries_dev || !out_ids_dev || !out_dists_dev || nq < 1 || K < 1 || K > L || L > 256 || W < 1 ||
+      W > 16 || (u64)W * ix->desc.max_degree > 1024)
+    return fail(ix, GORIO_ERR_INVALID_ARG, "search: need 1 <= K <= L <= 256, 1 <= W <= 16, W*max_degree <= 1024");
+  if (!ix->cache_ready) return fail(ix, GORIO_ERR_STATE, "search: call gorio_cache_config first");
+  CK(cudaSetDevice(ix->dev));
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  const auto t_begin = Clock::now();
+  if (ix->cache_dirty) {           // a failed search left requests in flight: start from a clean cache
+    int st = setup_cache(ix);
+    if (st != GORIO_OK) return st;
+  }
+  int st = ensure_qstate(ix, nq, K, L, W);
+  if (st != GORIO_OK) return st;
+
+  const gorio_index_desc &d = ix->desc;
+  Ctx &c = ix->ctx;
+  c.n_nodes = (u32)d.n_nodes; c.dim = d.dim; c.dtype = d.dtype; c.R = d.max_degree; c.npp = d.nodes_per_page;
+  c.node_bytes = ix->node_bytes; c.vec_bytes = ix->vec_bytes; c.entry = d.entry_id; c.n_pages = ix->n_pages;
+  c.pq_m = d.pq_m; c.pq_dsub = d.pq_m ? d.dim / d.pq_m : 0; c.pq_cent = d.pq_centroids_dev; c.pq_codes = d.pq_codes_dev;
+  c.slot_data = ix->slot_data; c.tag = ix->tag; c.wl = ix->wl; c.hand = ix->hand;
+  c.n_sets = ix->n_sets; c.n_slots = ix->n_slots;
+  c.ring = ix->ring_d; c.ring_mask = ix->ring_cap - 1; c.ring_shift = ilog2(ix->ring_cap);
+  c.comp_ring = ix->comp_d; c.comp_mask = ix->ring_cap - 1; c.host_ctl = ix->hctl_d;
+  c.ctl = ix->ctl;
+  c.arr = Queue{(u32 *)ix->arr_buf, ix->ring_cap - 1, &ix->ctl->q_heads[0], &ix->ctl->q_heads[1]};
+  c.run = Queue{(u32 *)ix->run_buf, ix->runq_cap - 1, &ix->ctl->q_heads[2], &ix->ctl->q_heads[3]};
+  c.retry = Queue{(u32 *)ix->retry_buf, ix->runq_cap - 1, &ix->ctl->q_heads[4], &ix->ctl->q_heads[5]};
+  c.nq = nq; c.K = K; c.L = L; c.W = W; c.WR = ix->qs_WR;
+  c.queries = queries_dev; c.out_ids = out_ids_dev; c.out_dists = out_dists_dev;
+  c.out_pages = out_pages_distinct_dev; c.out_counters = out_counters_dev;
+  c.timeout_ns = (u64)ix->cfg.timeout_ms * 1000000ull;
+  c.max_iters = 64u * L + 1024u;
+
+  // launch geometry: leave room on every SM for the proxy's copy kernels
+  const bool pq = d.pq_m != 0;
+  u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 6u : 16u);
+  if (pq) { u32 lim = (200u * 1024u) / (d.pq_m * kPqKsub * 4u); if (warps > lim) warps = lim; }
+  if (warps < 2) return fail(ix, GORIO_ERR_INVALID_ARG, "search: shared memory cannot hold two PQ tables per block");
+  int occ = 0;
+  CK(search_occupancy(pq, warps, &occ));
+  if (occ < 1) return fail(ix, GORIO_ERR_INVALID_ARG, "search: launch geometry does not fit an SM");
+  u32 bps = ix->tune.blocks_per_sm ? ix->tune.blocks_per_sm : 1u;
+  if ((int)bps > occ) bps = (u32)occ;
+  const u32 blocks = (u32)ix->n_sms * bps;
+
+  // reset the host-visible rings while the proxy is idle
+  std::memset(ix->ring_h, 0, (size_t)ix->ring_cap * 8);
+  std::memset(ix->hctl_h, 0, 64 * 4);
+  std::atomic_thread_fence(std::memory_order_seq_cst);
+
+  CK(cudaMemsetAsync(c.seen, 0xFF, (size_t)c.n_qslots * c.seen_cap * 4, stream));
+  CK(cudaMemsetAsync(c.pset, 0xFF, (size_t)c.n_qslots * c.pset_cap * 4, stream));
+  CK(launch_init(c, stream));
+  ix->cache_dirty = true;      // until this search ends cleanly
+  proxy_start(ix);
+  cudaError_t le = launch_search(c, blocks, warps, stream);
+  if (le != cudaSuccess) { proxy_stop(ix); return cuda_fail(ix, le, "launch_search"); }
+  cudaEventRecord(ix->done_ev, stream);
+
+  // wait for the kernel; a host-side watchdog asks the device to abort if it overruns
+  const auto deadline = Clock::now() + std::chrono::milliseconds(ix->cfg.timeout_ms);
+  bool host_abort = false;
+  cudaError_t qe;
+  while ((qe = cudaEventQuery(ix->done_ev)) == cudaErrorNotReady) {
+    if (ix->px_error.load() && !host_abort) { ((volatile u32 *)ix->hctl_h)[1] = 1; host_abort = true; }
+    if (!host_abort && Clock::now() > deadline) { ((volatile u32 *)ix->hctl_h)[1] = 1; host_abort = true; }
+    std::this_thread::sleep_for(std::chrono::microseconds(20));
+  }
+  proxy_stop(ix);
+  for (int i = 0; i < kMaxFillStreams; ++i) cudaStreamSynchronize(ix->fill_streams[i]);
+  if (qe != cudaSuccess) return cuda_fail(ix, qe, "search kernel");
+  Ctl h{};
+  CK(cudaMemcpyAsync(&h, ix->ctl, sizeof(Ctl), cudaMemcpyDeviceToHost, stream));
+  CK(cudaStreamSynchronize(stream));
+  ix->host_search_ns += (u64)std::chrono::duration_cast<std::chrono::nanoseconds>(Clock::now() - t_begin).count();
+  if (ix->px_error.load()) return fail(ix, GORIO_ERR_INTERNAL, "proxy: bad descriptor or copy launch failure");
+  if (h.status != 0 || h.stop != 1) {
+    char buf[640];
+    const u32 s = h.status ? h.status : (u32)GORIO_ERR_INTERNAL;
+    std::snprintf(buf, sizeof buf,
+                  "device: %s (site 0x%x, %u, %u, %u; block %u thread %u; done %u/%u; posted %u; arrivals %u/%u; "
+                  "runnable %u/%u; retry %u/%u; proxy consumed %u published %u outstanding %u queued %u "
+                  "[head stream %u seq %u copied %u])",
+                  s < 9 ? kDeviceErr[s] : "?", h.dbg[0], h.dbg[1], h.dbg[2], h.dbg[3], h.dbg[4], h.dbg[5], h.done, nq,
+                  h.ring_head, h.q_heads[0], h.q_heads[1], h.q_heads[2], h.q_heads[3], h.q_heads[4], h.q_heads[5],
+                  ix->px_dbg[0], ix->px_dbg[1], ix->px_dbg[2], ix->px_dbg[3], ix->px_dbg[4], ix->px_dbg[5], ix->px_dbg[6]);
+    return fail(ix, (int)s, buf);
+  }
+  ix->cache_dirty = false;
+  return GORIO_OK;
+}
+
+int gorio_search_host(gorio_index *ix, const void *queries_host, uint32_t nq, uint32_t K, uint32_t L, uint32_t W,
+                      uint32_t *out_ids_host, void *out_dists_host, uint32_t *out_pages_distinct_host,
+                      uint32_t *out_counters_host) {
+  if (!ix || !queries_host || !out_ids_host || !out_dists_host || nq < 1 || K < 1) return GORIO_ERR_INVALID_ARG;
+  CK(cudaSetDevice(ix->dev));
+  const size_t qb = (size_t)nq * ix->vec_bytes;
+  const size_t ob = (size_t)nq * K * 8 + (size_t)nq * 4 + (size_t)nq * 20;
+  if (qb > ix->st_q_bytes) { cudaFree(ix->st_q); ix->st_q = nullptr; CK(cudaMalloc(&ix->st_q, qb)); ix->st_q_bytes = qb; }
+  if (ob > ix->st_out_bytes) { cudaFree(ix->st_out); ix->st_out = nullptr; CK(cudaMalloc(&ix->st_out, ob)); ix->st_out_bytes = ob; }
+  u32 *ids = (u32 *)ix->st_out;
+  u32 *dists = ids + (size_t)nq * K;
+  u32 *pages = dists + (size_t)nq * K;
+  u32 *counters = pages + nq;
+  cudaStream_t s = ix->own_stream;
+  CK(cudaMemcpyAsync(ix->st_q, queries_host, qb, cudaMemcpyHostToDevice, s));
+  int st = gorio_search(ix, ix->st_q, nq, K, L, W, ids, dists, pages, counters, s);
+  if (st != GORIO_OK) return st;
+  CK(cudaMemcpyAsync(out_ids_host, ids, (size_t)nq * K * 4, cudaMemcpyDeviceToHost, s));
+  CK(cudaMemcpyAsync(out_dists_host, dists, (size_t)nq * K * 4, cudaMemcpyDeviceToHost, s));
+  if (out_pages_distinct_host) CK(cudaMemcpyAsync(out_pages_distinct_host, pages, (size_t)nq * 4, cudaMemcpyDeviceToHost, s));
+  if (out_counters_host) CK(cudaMemcpyAsync(out_counters_host, counters, (size_t)nq * 20, cudaMemcpyDeviceToHost, s));
+  CK(cudaStreamSynchronize(s));
+  return GORIO_OK;
+}
+
+int gorio_stats(gorio_index *ix, gorio_stats_t *out) {
+  if (!ix || !out) return GORIO_ERR_INVALID_ARG;
+  CK(cudaSetDevice(ix->dev));
+  Ctl h{};
+  CK(cudaMemcpy(&h, ix->ctl, sizeof(Ctl), cudaMemcpyDeviceToHost));
+  std::memset(out, 0, sizeof(*out));
+  out->pages_hit = h.stats[S_HIT]; out->pages_missed = h.stats[S_MISSED]; out->pages_fetched = ix->host_fetched;
+  out->dedupe_joins = h.stats[S_JOINS]; out->evictions = h.stats[S_EVICT]; out->retries = h.stats[S_RETRY];
+  out->max_outstanding_seen = ix->host_max_out; out->queries_done = h.stats[S_DONE];
+  out->n_eval = h.stats[S_NEVAL]; out->n_expand = h.stats[S_NEXPAND]; out->sum_degree = h.stats[S_SUMDEG];
+  out->n_iter = h.stats[S_NITER]; out->resumes = h.stats[S_RESUMES]; out->search_ns = ix->host_search_ns;
+  out->proxy_batches = ix->host_batches; out->reserved0 = h.stats[S_POSTED];
+  return GORIO_OK;
+}
+
+int gorio_stats_reset(gorio_index *ix) {
+  if (!ix) return GORIO_ERR_INVALID_ARG;
+  CK(cudaSetDevice(ix->dev));
+  CK(cudaMemset((u8 *)ix->ctl + offsetof(Ctl, stats), 0, sizeof(((Ctl *)0)->stats)));
+  ix->host_fetched = ix->host_max_out = ix->host_batches = ix->host_search_ns = 0;
+  return GORIO_OK;
+}
+
+}  // extern "C"

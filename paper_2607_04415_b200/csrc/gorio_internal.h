@@ -1,0 +1,127 @@
+// Internal definitions shared by the host API (gorio_api.cu) and the device code
+// (search_kernels.cu).  Nothing here is part of the public C ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace gorio {
+
+typedef uint8_t u8;
+typedef uint16_t u16;
+typedef uint32_t u32;
+typedef uint64_t u64;
+
+constexpr u32 kPageBytes = 4096;
+constexpr u32 kWays = 16;             // set associativity of the page cache
+constexpr u32 kNil = 0xFFFFFFFFu;     // end of a waiter list
+constexpr u32 kClosed = 0xFFFFFFFEu;  // waiter list closed: the page has arrived
+constexpr u32 kInvalidId = 0xFFFFFFFFu;
+constexpr u64 kPadKey = ~0ull;        // sorts after every real key
+constexpr u32 kMaxFillBatch = 128;
+constexpr u32 kPqKsub = 256;
+
+// Slot tag word: [page:32][generation:28][ref:1][state:3]
+enum SlotState : u32 { ST_EMPTY = 0, ST_RESERVED = 1, ST_FILLING = 2, ST_ARRIVED = 3, ST_READY = 4 };
+
+// Query phases: which batch of page items is outstanding for the query slot.
+enum Phase : u32 { PH_NEW = 0, PH_EVAL = 1, PH_EXPAND = 2 };
+
+// Per-query-slot header (64 bytes).  Written by the warp that runs the query; `awaiting`
+// is decremented by whoever consumes one of the query's page items.
+struct QHdr {
+  u32 qid;
+  u32 phase;
+  u32 awaiting;   // outstanding items of the current batch (+1 guard while issuing/retrying)
+  u32 n_items;    // items in the current batch
+  u32 n_todo;     // items of the batch whose lookup must be retried
+  u32 list_len;
+  u32 n_iter, n_expand, n_eval, sum_deg, pages_distinct;
+  u32 pool_len;   // PQ mode: entries in the rerank pool
+  u32 pad[4];
+};
+
+// Multi-producer multi-consumer ring of u32 values in HBM (cells hold value+1, 0 = empty).
+struct Queue {
+  u32 *buf;
+  u32 mask;
+  u32 *head;
+  u32 *tail;
+};
+
+// Device-resident control block.
+struct Ctl {
+  u32 stop;        // 0 run, 1 all queries done, 2 error/abort
+  u32 status;      // first gorio_status raised on the device
+  u32 next_query;  // next query id to admit when a slot frees
+  u32 done;        // queries finished
+  u32 ring_head;   // request descriptors posted
+  u32 q_heads[8];  // queue head/tail words: arr(0,1) run(2,3) retry(4,5)
+  u32 dbg[8];      // detail of the first error
+  u64 stats[16];
+};
+
+enum StatIdx { S_HIT = 0, S_MISSED, S_JOINS, S_EVICT, S_RETRY, S_DONE, S_NEVAL, S_NEXPAND,
+               S_SUMDEG, S_NITER, S_RESUMES, S_POSTED };
+
+// Everything the persistent kernel needs, passed by value.
+struct Ctx {
+  // index
+  u32 n_nodes, dim, dtype, R, npp, node_bytes, vec_bytes, entry, n_pages;
+  u32 pq_m, pq_dsub;
+  const u8 *pq_cent;
+  const u8 *pq_codes;
+  // page cache
+  u8 *slot_data;   // n_slots * 4096, slot = way * n_sets + set
+  u64 *tag;        // [n_sets][kWays]
+  u64 *wl;         // [n_sets][kWays]  (generation << 32 | waiter list head)
+  u32 *hand;       // [n_sets] clock hands
+  u32 n_sets, n_slots;
+  // miss ring: host-mapped, written by the GPU, consumed by the proxy
+  u64 *ring;
+  u32 ring_mask, ring_shift;
+  // completions: host-mapped, written by the proxy, polled by the GPU
+  const u32 *comp_ring;
+  u32 comp_mask;
+  const u32 *host_ctl;  // [0] completion tail, [1] abort request
+  Queue arr, run, retry;
+  // query state
+  u32 n_qslots, nq, K, L, W, WR;
+  QHdr *hdr;
+  u64 *list;     // [n_qslots][L]
+  u64 *cand;     // [n_qslots][WR]
+  u32 *items;    // [n_qslots][WR] node id of each item of the current batch
+  u32 *wrec;     // [n_qslots][WR] next pointers of waiter records (record id = qs*WR + j)
+  u32 *adj;      // [n_qslots][W][R]
+  u32 *adjdeg;   // [n_qslots][W]
+  u16 *todo;     // [n_qslots][WR]
+  u32 *seen;     // [n_qslots][seen_cap]
+  u32 *pset;     // [n_qslots][pset_cap]
+  u64 *pool;     // [n_qslots][K + W]   PQ rerank pool (sorted, <= K kept)
+  u32 seen_cap, pset_cap;
+  const void *queries;
+  u32 *out_ids;
+  void *out_dists;
+  u32 *out_pages;
+  u32 *out_counters;
+  Ctl *ctl;
+  u64 timeout_ns;
+  u32 max_iters;
+};
+
+struct FillBatch {
+  u32 n;
+  u32 seq;
+  u32 page[kMaxFillBatch];
+  u32 slot[kMaxFillBatch];
+};
+
+// launchers implemented in search_kernels.cu
+cudaError_t preload_kernels();
+cudaError_t launch_init(const Ctx &c, cudaStream_t s);
+cudaError_t launch_search(const Ctx &c, u32 blocks, u32 warps_per_block, cudaStream_t s);
+cudaError_t search_occupancy(bool pq, u32 warps_per_block, int *blocks_per_sm);
+cudaError_t launch_fill(const FillBatch &b, const u8 *host_pages_dev, u8 *slot_data,
+                        u32 *counter, u32 *host_copied, cudaStream_t s);
+cudaError_t launch_cache_reset(const Ctx &c, u32 preloaded_pages, cudaStream_t s);
+
+}  // namespace gorio

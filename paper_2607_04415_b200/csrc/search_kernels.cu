@@ -1,0 +1,982 @@
+// Device side of the GPU-owned paged beam search (sm_100a).
+//
+// One persistent kernel runs every query of a batch.  Warps are the execution slots: a
+// warp pops a runnable query slot from a queue in HBM, advances it by one or more phases,
+// and parks it when it has to wait for pages (paper Section 3.3: blocks "claim work,
+// execute graph traversal, and either finish a query or mark it pending on a missing page").
+//
+// Data flow of one query iteration:
+//   PH_EVAL  complete -> merge the scored candidates into the sorted L-entry list, pick the
+//                        first W unexpanded entries (the frontier), issue their pages
+//   PH_EXPAND complete -> read the frontier's adjacency lists, filter through the exact
+//                        visited set, issue the pages of the new neighbours (exact mode) or
+//                        score them from resident PQ codes (PQ mode)
+// "Issuing" a batch of page items means, per item: look the page up in the cache; on a hit
+// consume it now; if the page is in flight register as a waiter; if it is absent claim a
+// slot (clock eviction), post a request descriptor to the host-visible ring and register.
+// A page that arrives is consumed for every registered waiter by whichever warp picks the
+// arrival up, using only the waiter's query vector, so no page stays pinned for a query.
+// The last item consumed of a batch pushes the query back onto the runnable queue.
+#include "gorio_internal.h"
+
+namespace gorio {
+
+// ------------------------------------------------------------------------------------------
+// memory access helpers: query/cache state is shared between SMs, so it is always read and
+// written at the L2 (relaxed, gpu scope); host-mapped words use system scope.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ u32 ld_u32(const u32 *p) {
+  u32 v; asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory"); return v;
+}
+__device__ __forceinline__ u64 ld_u64(const u64 *p) {
+  u64 v; asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory"); return v;
+}
+__device__ __forceinline__ u16 ld_u16(const u16 *p) {
+  u16 v; asm volatile("ld.relaxed.gpu.global.u16 %0, [%1];" : "=h"(v) : "l"(p) : "memory"); return v;
+}
+__device__ __forceinline__ void st_u32(u32 *p, u32 v) {
+  asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void st_u64(u64 *p, u64 v) {
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ void st_u16(u16 *p, u16 v) {
+  asm volatile("st.relaxed.gpu.global.u16 [%0], %1;" ::"l"(p), "h"(v) : "memory");
+}
+__device__ __forceinline__ u32 ld_sys_u32(const u32 *p) {
+  u32 v; asm volatile("ld.relaxed.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory"); return v;
+}
+__device__ __forceinline__ void st_sys_u64(u64 *p, u64 v) {
+  asm volatile("st.relaxed.sys.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ void fence_sc() { asm volatile("fence.sc.gpu;" ::: "memory"); }
+__device__ __forceinline__ u64 globaltimer() {
+  u64 t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t;
+}
+__device__ __forceinline__ u32 lane_id() { return threadIdx.x & 31u; }
+
+// ------------------------------------------------------------------------------------------
+// errors and statistics
+// ------------------------------------------------------------------------------------------
+__device__ __noinline__ void raise(const Ctx &c, u32 status, u32 a = 0, u32 b = 0, u32 d = 0, u32 e = 0) {
+  if (atomicCAS(&c.ctl->status, 0u, status) == 0u) {
+    c.ctl->dbg[0] = a; c.ctl->dbg[1] = b; c.ctl->dbg[2] = d; c.ctl->dbg[3] = e;
+    c.ctl->dbg[4] = blockIdx.x; c.ctl->dbg[5] = threadIdx.x;
+    __threadfence();
+  }
+  st_u32(&c.ctl->stop, 2u);
+}
+__device__ __forceinline__ bool stopped(const Ctx &c) { return ld_u32(&c.ctl->stop) != 0u; }
+// warp-uniform variants: every lane gets lane 0's view, and the shuffle is a convergence point
+__device__ __forceinline__ bool warp_stopped(const Ctx &c) {
+  return __shfl_sync(0xffffffffu, ld_u32(&c.ctl->stop), 0) != 0u;
+}
+__device__ __forceinline__ u32 uld(const u32 *p) { return __shfl_sync(0xffffffffu, ld_u32(p), 0); }
+__device__ __forceinline__ void stat_add(const Ctx &c, u32 idx, u32 v) {
+  if (v) atomicAdd((unsigned long long *)&c.ctl->stats[idx], (unsigned long long)v);
+}
+
+// ------------------------------------------------------------------------------------------
+// bounded MPMC queue of u32 (cells = sequence << 32 | value); one lane calls these
+// ------------------------------------------------------------------------------------------
+constexpr u32 kSpinLimit = 1u << 22;
+
+__device__ void q_push(const Ctx &c, const Queue &q, u32 v) {
+  __threadfence();   // everything written for the consumer is visible before the cell
+  u32 pos = atomicAdd(q.tail, 1u);
+  u64 *cell = (u64 *)q.buf + (pos & q.mask);
+  u32 spins = 0;
+  while ((u32)(ld_u64(cell) >> 32) != pos) {      // previous lap's consumer not done yet
+    if (++spins > kSpinLimit) { raise(c, 8, 0x51, pos); return; }
+  }
+  st_u64(cell, ((u64)(pos + 1u) << 32) | v);
+}
+
+__device__ bool q_pop(const Ctx &c, const Queue &q, u32 &out) {
+  for (int tries = 0; tries < 8; ++tries) {
+    u32 h = ld_u32(q.head), t = ld_u32(q.tail);
+    if ((int)(t - h) <= 0) return false;
+    if (atomicCAS(q.head, h, h + 1u) != h) continue;
+    u64 *cell = (u64 *)q.buf + (h & q.mask);
+    u32 spins = 0;
+    u64 v;
+    while ((u32)((v = ld_u64(cell)) >> 32) != h + 1u) {
+      if (++spins > kSpinLimit) { raise(c, 8, 0x52, h); return false; }
+    }
+    st_u64(cell, (u64)(h + q.mask + 1u) << 32);
+    __threadfence();
+    out = (u32)v;
+    return true;
+  }
+  return false;
+}
+
+// warp-level pop: lane 0 pops, the result is broadcast
+__device__ __forceinline__ bool warp_pop(const Ctx &c, const Queue &q, u32 &out, u32 lane) {
+  u32 ok = 0, v = 0;
+  if (lane == 0) ok = q_pop(c, q, v) ? 1u : 0u;
+  ok = __shfl_sync(0xffffffffu, ok, 0);
+  out = __shfl_sync(0xffffffffu, v, 0);
+  return ok != 0u;
+}
+
+// ------------------------------------------------------------------------------------------
+// slot tags
+// ------------------------------------------------------------------------------------------
+constexpr u64 kRefBit = 8ull;
+__device__ __forceinline__ u64 mk_tag(u32 page, u32 gen, u32 ref, u32 state) {
+  return ((u64)page << 32) | ((u64)(gen & 0x0FFFFFFFu) << 4) | ((u64)ref << 3) | state;
+}
+__device__ __forceinline__ u32 tag_page(u64 t) { return (u32)(t >> 32); }
+__device__ __forceinline__ u32 tag_gen(u64 t) { return (u32)(t >> 4) & 0x0FFFFFFFu; }
+__device__ __forceinline__ u32 tag_state(u64 t) { return (u32)t & 7u; }
+__device__ __forceinline__ u32 slot_of(const Ctx &c, u32 ti) { return (ti % kWays) * c.n_sets + ti / kWays; }
+__device__ __forceinline__ u32 ti_of(const Ctx &c, u32 slot) { return (slot % c.n_sets) * kWays + slot / c.n_sets; }
+
+// lookup result: [gen:28 | pad][ti:29][code:3]
+enum LookupCode : u32 { LK_NONE = 0, LK_HIT = 1, LK_WAIT = 2, LK_DEFER = 3 };
+__device__ __forceinline__ u64 mk_res(u32 code, u32 ti, u32 gen) { return ((u64)gen << 32) | ((u64)ti << 3) | code; }
+
+struct LaneStats { u32 hit, missed, joins, evict, retry, posted; };
+
+// Post a request descriptor: one 64-bit word [page:32][slot:24][lap:8] in host-mapped memory.
+// The ring holds at least twice as many entries as there are slots, and every pending
+// request owns a distinct FILLING slot, so an entry is never overwritten before the proxy
+// has consumed it.  (Section 3.2: reserve a descriptor slot atomically, record page id and
+// target cache slot, publish through a ready flag -- here the lap tag inside the word.)
+__device__ __forceinline__ void post_request(const Ctx &c, u32 page, u32 slot) {
+  u32 idx = atomicAdd(&c.ctl->ring_head, 1u);
+  u32 lap = ((idx >> c.ring_shift) % 255u) + 1u;
+  st_sys_u64(c.ring + (idx & c.ring_mask), ((u64)page << 32) | ((u64)slot << 8) | lap);
+}
+
+// Page lookup / miss generation by ONE lane (lanes of a warp that want the same page elect a
+// leader first, so a warp never races with itself).
+__device__ u64 cache_lookup(const Ctx &c, u32 page, LaneStats &st) {
+  const u32 set = page % c.n_sets;
+  u64 *tags = c.tag + (u64)set * kWays;
+  for (int attempt = 0; attempt < 24; ++attempt) {
+    // 1. scan the set
+    int found = -1; u64 ft = 0;
+#pragma unroll
+    for (int w = 0; w < (int)kWays; ++w) {
+      u64 t = ld_u64(tags + w);
+      if (tag_page(t) == page && tag_state(t) != ST_EMPTY && found < 0) { found = w; ft = t; }
+    }
+    if (found >= 0) {
+      u32 s = tag_state(ft), ti = set * kWays + found;
+      if (s == ST_READY || s == ST_ARRIVED) return mk_res(LK_HIT, ti, tag_gen(ft));
+      if (s == ST_FILLING) return mk_res(LK_WAIT, ti, tag_gen(ft));
+      __nanosleep(64);           // RESERVED: another lane is deciding a race on this page
+      continue;
+    }
+    // 2. miss: claim a victim with the set's clock hand
+    // The page's home way ((page / n_sets) % ways) is tried first while it is empty: rival
+    // claims for one page then meet on a single compare-and-swap, and with capacity for
+    // every page each page has a way of its own, so nothing is ever evicted or fetched twice.
+    int victim = -1; u32 vgen = 0;
+    {
+      const u32 w = (page / c.n_sets) % kWays;
+      const u64 t = ld_u64(tags + w);
+      if (tag_state(t) == ST_EMPTY) {
+        const u64 nt = mk_tag(page, tag_gen(t) + 1u, 0, ST_RESERVED);
+        if (atomicCAS((unsigned long long *)(tags + w), t, nt) != t) continue;   // lost the race: rescan
+        victim = (int)w; vgen = tag_gen(nt);
+      } else if (tag_page(t) == page) {
+        continue;                                   // the page appeared meanwhile: rescan
+      }
+    }
+    // otherwise the set's clock hand picks a victim: second chance for referenced pages
+    for (int step = 0; victim < 0 && step < 3 * (int)kWays; ++step) {
+      const u32 w = atomicAdd(c.hand + set, 1u) % kWays;
+      const u64 t = ld_u64(tags + w);
+      const u32 s = tag_state(t);
+      if (s == ST_EMPTY || (s == ST_READY && !(t & kRefBit))) {
+        const u64 nt = mk_tag(page, tag_gen(t) + 1u, 0, ST_RESERVED);
+        if (atomicCAS((unsigned long long *)(tags + w), t, nt) == t) {
+          victim = (int)w; vgen = tag_gen(nt);
+          if (s == ST_READY) st.evict++;
+        }
+      } else if (s == ST_READY) {
+        atomicCAS((unsigned long long *)(tags + w), t, t & ~kRefBit);
+      }
+    }
+    if (victim < 0) return mk_res(LK_DEFER, 0, 0);     // every way is in flight: retry later
+    // 3. another lane may have claimed a way for the same page concurrently: whoever sees
+    //    a rival backs off, so at most one claim per page survives
+    fence_sc();
+    bool rival = false;
+#pragma unroll
+    for (int w = 0; w < (int)kWays; ++w) {
+      u64 t = ld_u64(tags + w);
+      if (w != victim && tag_page(t) == page && tag_state(t) != ST_EMPTY) rival = true;
+    }
+    const u32 ti = set * kWays + (u32)victim;
+    if (rival) {
+      st_u64(tags + victim, mk_tag(kInvalidId, vgen, 0, ST_EMPTY));
+      __nanosleep(32 + 16 * (lane_id() & 7u));
+      continue;
+    }
+    // 4. won: open the waiter list, publish FILLING, post the descriptor
+    st_u64(c.wl + ti, ((u64)vgen << 32) | kNil);
+    __threadfence();
+    st_u64(tags + victim, mk_tag(page, vgen, 0, ST_FILLING));
+    __threadfence_system();      // the tag must be visible to whoever learns of the request
+    post_request(c, page, slot_of(c, ti));
+    st.posted++;
+    return mk_res(LK_WAIT, ti, vgen) | (1ull << 63);    // bit 63: this lane is the owner
+  }
+  return mk_res(LK_DEFER, 0, 0);
+}
+
+// Link waiter record g (= query slot * WR + item) into the slot's list.
+__device__ bool register_waiter(const Ctx &c, u32 ti, u32 gen, u32 g) {
+  u64 *wl = c.wl + ti;
+  for (int tries = 0; tries < 128; ++tries) {
+    u64 cur = ld_u64(wl);
+    if ((u32)(cur >> 32) != gen || (u32)cur == kClosed) return false;
+    st_u32(c.wrec + g, (u32)cur);
+    __threadfence();
+    if (atomicCAS((unsigned long long *)wl, cur, ((u64)gen << 32) | g) == cur) return true;
+  }
+  return false;
+}
+
+// ------------------------------------------------------------------------------------------
+// distances (warp cooperative)
+// ------------------------------------------------------------------------------------------
+// Squared L2 between query qid and the vector at `rec` (a node record inside a cache slot).
+// uint8: per-lane 4-byte words, |a-b| per byte then a 4-way dot product into u32 (exact).
+// fp32 : per-lane strided elements, fused multiply-add, butterfly reduction (fixed order).
+__device__ __forceinline__ u32 warp_dist(const Ctx &c, const u8 *rec, u32 qid, u32 lane) {
+  const u8 *q = (const u8 *)c.queries + (u64)qid * c.vec_bytes;
+  if (c.dtype == 0) {
+    const u32 words = c.dim >> 2;
+    u32 acc = 0;
+    for (u32 w = lane; w < words; w += 32) {
+      u32 a = __ldcg((const u32 *)rec + w), b = __ldg((const u32 *)q + w);
+      u32 d = __vabsdiffu4(a, b);
+      acc = __dp4a(d, d, acc);
+    }
+    return __reduce_add_sync(0xffffffffu, acc);
+  } else {
+    float acc = 0.f;
+    for (u32 i = lane; i < c.dim; i += 32) {
+      float diff = __ldg((const float *)q + i) - __ldcg((const float *)rec + i);
+      acc = fmaf(diff, diff, acc);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    return __float_as_uint(acc);
+  }
+}
+__device__ __forceinline__ u64 mk_key(u32 dist, u32 id) { return ((u64)dist << 32) | ((u64)id << 1); }
+__device__ __forceinline__ u32 key_id(u64 k) { return (u32)(k & 0xFFFFFFFFull) >> 1; }
+__device__ __forceinline__ u32 key_dist(u64 k) { return (u32)(k >> 32); }
+
+// Consume item j of query slot qs from the page in `slot` (warp cooperative).
+//   PH_EVAL   : score the node, write its key into the candidate buffer.
+//   PH_EXPAND : copy the node's adjacency list into the query's buffer (PQ mode: also the
+//               node's exact distance into the rerank pool's staging entries).
+__device__ void consume_item(const Ctx &c, u32 qs, u32 j, u32 slot, u32 lane) {
+  const QHdr *h = c.hdr + qs;
+  const u32 phase = ld_u32(&h->phase), qid = ld_u32(&h->qid);
+  const u32 node = ld_u32(c.items + (u64)qs * c.WR + j);
+  const u8 *rec = c.slot_data + (u64)slot * kPageBytes + (node % c.npp) * c.node_bytes;
+  if (phase == PH_EVAL) {
+    u32 d = warp_dist(c, rec, qid, lane);
+    if (lane == 0) st_u64(c.cand + (u64)qs * c.WR + j, mk_key(d, node));
+  } else {
+    const u32 *adj = (const u32 *)(rec + c.vec_bytes);
+    u32 deg = __ldcg(adj);
+    u32 *dst = c.adj + ((u64)qs * c.W + j) * c.R;
+    for (u32 i = lane; i < c.R; i += 32) st_u32(dst + i, __ldcg(adj + 1 + i));
+    if (lane == 0) st_u32(c.adjdeg + (u64)qs * c.W + j, deg);
+    if (c.pq_m) {
+      u32 d = warp_dist(c, rec, qid, lane);
+      if (lane == 0) st_u64(c.pool + (u64)qs * (c.K + c.W) + c.K + j, mk_key(d, node));
+    }
+  }
+}
+
+// n items of query slot qs are done; the one that brings `awaiting` to zero resumes it.
+__device__ __forceinline__ void complete_items(const Ctx &c, u32 qs, u32 n) {
+  __threadfence();
+  u32 old = atomicSub(&c.hdr[qs].awaiting, n);
+  if (old == n) { q_push(c, c.run, qs); stat_add(c, S_RESUMES, 1); }
+  else if (old < n) raise(c, 8, 0x61, qs, old, n);
+}
+
+// A page has arrived in `slot`: consume it for every registered waiter, then make it
+// evictable.  (Section 3.2: the per-slot ready entry is what the GPU tests on resume.)
+__device__ void consume_arrival(const Ctx &c, u32 slot, u32 lane) {
+  if (slot >= c.n_slots) { if (lane == 0) raise(c, 8, 0x71, slot); return; }
+  const u32 ti = ti_of(c, slot);
+  u64 t = ld_u64(c.tag + ti);
+  t = __shfl_sync(0xffffffffu, t, 0);
+  if (tag_state(t) != ST_FILLING) { if (lane == 0) raise(c, 8, 0x72, slot, (u32)t, (u32)(t >> 32)); return; }
+  const u32 page = tag_page(t), gen = tag_gen(t);
+  u32 head = 0;
+  if (lane == 0) {
+    st_u64(c.tag + ti, mk_tag(page, gen, 1, ST_ARRIVED));
+    __threadfence();
+    u64 old = atomicExch((unsigned long long *)(c.wl + ti), ((u64)gen << 32) | kClosed);
+    head = (u32)old;
+    __threadfence();
+  }
+  head = __shfl_sync(0xffffffffu, head, 0);
+  u32 g = head, count = 0;
+  const u32 limit = c.n_qslots * c.WR;
+  while (g != kNil) {
+    if (g >= limit || ++count > limit) { if (lane == 0) raise(c, 8, 0x73, slot, g, count); return; }
+    const u32 next = ld_u32(c.wrec + g);
+    const u32 qs = g / c.WR, j = g % c.WR;
+    consume_item(c, qs, j, slot, lane);
+    __threadfence();      // every lane's result stores before lane 0 counts the item done
+    __syncwarp();
+    if (lane == 0) complete_items(c, qs, 1);
+    g = next;
+  }
+  __syncwarp();
+  if (lane == 0) { __threadfence(); st_u64(c.tag + ti, mk_tag(page, gen, 1, ST_READY)); }
+}
+
+// ------------------------------------------------------------------------------------------
+// per-query exact sets (open addressing, linear probing, 0xFFFFFFFF = empty)
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ u32 hash32(u32 v) { v *= 0x9E3779B1u; v ^= v >> 15; return v * 0x85EBCA77u; }
+
+// returns 1 if v was inserted now, 0 if already present, 2 if the table is full
+__device__ u32 set_insert(u32 *tab, u32 cap, u32 v) {
+  u32 h = hash32(v) & (cap - 1);
+  for (u32 p = 0; p < cap; ++p) {
+    u32 old = atomicCAS(tab + h, kInvalidId, v);
+    if (old == kInvalidId) return 1;
+    if (old == v) return 0;
+    h = (h + 1) & (cap - 1);
+  }
+  return 2;
+}
+
+// ------------------------------------------------------------------------------------------
+// issue a batch of page items for query slot qs
+// ------------------------------------------------------------------------------------------
+// from_todo = false: items 0..n_items-1 of the current batch, `awaiting` is armed here.
+// from_todo = true : retry the deferred items listed in todo[0..n_todo).
+// Returns true if the whole batch is complete (the caller goes on inline); false if the
+// query was parked (someone else resumes it) or re-queued for a retry.
+__device__ bool issue_batch(const Ctx &c, u32 qs, bool from_todo, u32 lane) {
+  QHdr *h = c.hdr + qs;
+  const u32 phase = uld(&h->phase);
+  const u32 n = from_todo ? uld(&h->n_todo) : uld(&h->n_items);
+  const bool count_pages = !from_todo && ((c.pq_m == 0) == (phase == PH_EVAL));
+  if (!from_todo) {
+    if (lane == 0) st_u32(&h->awaiting, n + 1u);
+  }
+  __threadfence();
+  __syncwarp();
+  u16 *todo = c.todo + (u64)qs * c.WR;
+  const u32 *items = c.items + (u64)qs * c.WR;
+  u32 *pset = c.pset + (u64)qs * c.pset_cap;
+  LaneStats st = {0, 0, 0, 0, 0, 0};
+  u32 n_done = 0, n_todo_new = 0, new_pages = 0;
+
+  for (u32 base = 0; base < n; base += 32) {
+    const u32 idx = base + lane;
+    const bool active = idx < n;
+    u32 j = 0, node = 0, page = kInvalidId;
+    if (active) {
+      j = from_todo ? (u32)ld_u16(todo + idx) : idx;
+      node = ld_u32(items + j);
+      page = node / c.npp;
+      if (count_pages) {
+        u32 r = set_insert(pset, c.pset_cap, page);
+        if (r == 1) new_pages++;
+        else if (r == 2) raise(c, 6, 0x81, qs, page);
+      }
+    }
+    __syncwarp();
+    // lanes that want the same page elect the lowest lane as leader
+    const u32 amask = __ballot_sync(0xffffffffu, active);
+    u64 res = 0;
+    u32 leader = lane;
+    if (active) {
+      u32 grp = __match_any_sync(amask, page);
+      leader = __ffs(grp) - 1;
+      if (leader == lane) res = cache_lookup(c, page, st);
+    }
+    __syncwarp();
+    res = __shfl_sync(0xffffffffu, res, leader);
+    u32 code = active ? (u32)(res & 7u) : LK_NONE;
+    const u32 ti = (u32)((res & 0xFFFFFFFFull) >> 3), gen = (u32)(res >> 32) & 0x0FFFFFFFu;
+    const bool owner = (res >> 63) && leader == lane;
+    if (code == LK_WAIT) {
+      if (register_waiter(c, ti, gen, qs * c.WR + j)) { st.missed++; if (!owner) st.joins++; }
+      else code = LK_DEFER;
+    }
+    // hits: consume now (warp cooperative, one item at a time), then validate the tags
+    u32 hits = __ballot_sync(0xffffffffu, code == LK_HIT);
+    for (u32 m = hits; m; m &= m - 1) {
+      const u32 src = __ffs(m) - 1;
+      const u32 sj = __shfl_sync(0xffffffffu, j, src);
+      const u32 sti = __shfl_sync(0xffffffffu, ti, src);
+      consume_item(c, qs, sj, slot_of(c, sti), lane);
+    }
+    if (hits) {
+      __threadfence();
+      if (code == LK_HIT) {
+        u64 t2 = ld_u64(c.tag + ti);
+        const u32 s2 = tag_state(t2);
+        if (tag_page(t2) == page && tag_gen(t2) == gen && (s2 == ST_READY || s2 == ST_ARRIVED)) {
+          if (!(t2 & kRefBit)) atomicCAS((unsigned long long *)(c.tag + ti), t2, t2 | kRefBit);
+          st.hit++; n_done++;
+        } else {
+          code = LK_DEFER;     // evicted while we were reading: the item is redone later
+        }
+      }
+    }
+    // deferred items go (back) on the todo list; in-place compaction is safe because every
+    // lane has already read its entry of this round
+    __syncwarp();
+    const u32 defer = __ballot_sync(0xffffffffu, code == LK_DEFER);
+    if (code == LK_DEFER) {
+      st_u16(todo + n_todo_new + __popc(defer & ((1u << lane) - 1u)), (u16)j);
+      st.retry++;
+    }
+    n_todo_new += __popc(defer);
+    if (warp_stopped(c)) break;
+  }
+
+  // warp totals
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    n_done += __shfl_xor_sync(0xffffffffu, n_done, o);
+    new_pages += __shfl_xor_sync(0xffffffffu, new_pages, o);
+    st.hit += __shfl_xor_sync(0xffffffffu, st.hit, o);
+    st.missed += __shfl_xor_sync(0xffffffffu, st.missed, o);
+    st.joins += __shfl_xor_sync(0xffffffffu, st.joins, o);
+    st.evict += __shfl_xor_sync(0xffffffffu, st.evict, o);
+    st.retry += __shfl_xor_sync(0xffffffffu, st.retry, o);
+    st.posted += __shfl_xor_sync(0xffffffffu, st.posted, o);
+  }
+  u32 complete = 0;
+  __threadfence();
+  __syncwarp();
+  if (lane == 0) {
+    stat_add(c, S_HIT, st.hit); stat_add(c, S_MISSED, st.missed); stat_add(c, S_JOINS, st.joins);
+    stat_add(c, S_EVICT, st.evict); stat_add(c, S_RETRY, st.retry); stat_add(c, S_POSTED, st.posted);
+    if (new_pages) st_u32(&h->pages_distinct, ld_u32(&h->pages_distinct) + new_pages);
+    if (n_todo_new == 0) {
+      st_u32(&h->n_todo, 0);
+      __threadfence();
+      u32 old = atomicSub(&h->awaiting, n_done + 1u);       // drop the guard too
+      if (old == n_done + 1u) complete = 1;
+      else if (old < n_done + 1u) raise(c, 8, 0x82, qs, old, n_done);
+    } else {
+      st_u32(&h->n_todo, n_todo_new);
+      __threadfence();
+      if (n_done) {
+        u32 old = atomicSub(&h->awaiting, n_done);           // the guard stays
+        if (old <= n_done) raise(c, 8, 0x83, qs, old, n_done);
+      }
+      q_push(c, c.retry, qs);
+    }
+  }
+  return __shfl_sync(0xffffffffu, complete, 0) != 0u;
+}
+
+// ------------------------------------------------------------------------------------------
+// warp-sorted candidate list
+// ------------------------------------------------------------------------------------------
+// Bitonic sort of 32*NPL u64 keys held NPL per lane, element e at lane e%32, register e/32.
+template <int NPL>
+__device__ __forceinline__ void bitonic_sort(u64 (&x)[NPL], u32 lane) {
+#pragma unroll
+  for (int k = 2; k <= 32 * NPL; k <<= 1) {
+#pragma unroll
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      if (j >= 32) {
+        const int jr = j >> 5;
+#pragma unroll
+        for (int r = 0; r < NPL; ++r) {
+          const int pr = r ^ jr;
+          if (pr > r) {
+            const bool asc = ((r << 5) & k) == 0;
+            const u64 a = x[r], b = x[pr];
+            const bool sw = asc ? (a > b) : (a < b);
+            x[r] = sw ? b : a;
+            x[pr] = sw ? a : b;
+          }
+        }
+      } else {
+#pragma unroll
+        for (int r = 0; r < NPL; ++r) {
+          const u64 a = x[r];
+          const u64 b = __shfl_xor_sync(0xffffffffu, a, j);
+          const bool asc = ((((u32)r << 5) | lane) & (u32)k) == 0;
+          const bool lower = (lane & (u32)j) == 0;
+          const u64 mn = a < b ? a : b, mx = a < b ? b : a;
+          x[r] = (asc == lower) ? mn : mx;
+        }
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void write_result(const Ctx &c, u32 qid, u32 k, u64 key, bool valid) {
+  const u64 o = (u64)qid * c.K + k;
+  c.out_ids[o] = valid ? key_id(key) : kInvalidId;
+  u32 d = valid ? key_dist(key) : (c.dtype == 0 ? kInvalidId : 0x7F800000u);
+  ((u32 *)c.out_dists)[o] = d;
+}
+
+// Merge the scored candidates of the finished PH_EVAL batch into the list (top-L by key),
+// then choose and mark the frontier: the first W unexpanded entries in key order.  The
+// frontier's node ids become the items of the next (PH_EXPAND) batch.  Returns |frontier|;
+// 0 means the search of this query is over (exact mode: the results are written here).
+template <int NPL>
+__device__ __noinline__ u32 merge_select(const Ctx &c, u32 qs, u32 lane) {
+  QHdr *h = c.hdr + qs;
+  u32 len = uld(&h->list_len);
+  const u32 nc = uld(&h->n_items);
+  u64 *list = c.list + (u64)qs * c.L;
+  const u64 *cand = c.cand + (u64)qs * c.WR;
+  constexpr u32 CAP = 32u * NPL;
+  u64 x[NPL];
+#pragma unroll
+  for (int r = 0; r < NPL; ++r) {
+    const u32 e = (u32)r * 32u + lane;
+    x[r] = e < len ? ld_u64(list + e) : kPadKey;
+  }
+  u32 done = 0;
+  while (done < nc) {
+    const u32 take = min(CAP - len, nc - done);
+#pragma unroll
+    for (int r = 0; r < NPL; ++r) {
+      const u32 e = (u32)r * 32u + lane;
+      if (e >= len) x[r] = (e - len < take) ? ld_u64(cand + done + (e - len)) : kPadKey;
+    }
+    bitonic_sort<NPL>(x, lane);
+    len = min(c.L, len + take);
+    done += take;
+  }
+  // frontier
+  u32 taken = 0;
+  u32 *items = c.items + (u64)qs * c.WR;
+#pragma unroll
+  for (int r = 0; r < NPL; ++r) {
+    const u32 e = (u32)r * 32u + lane;
+    const bool un = e < len && !(x[r] & 1ull);
+    const u32 b = __ballot_sync(0xffffffffu, un);
+    if (taken < c.W && b) {
+      const u32 rank = taken + __popc(b & ((1u << lane) - 1u));
+      if (un && rank < c.W) { x[r] |= 1ull; st_u32(items + rank, key_id(x[r])); }
+      taken = min(c.W, taken + (u32)__popc(b));
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < NPL; ++r) {
+    const u32 e = (u32)r * 32u + lane;
+    if (e < len) st_u64(list + e, x[r]);
+  }
+  if (lane == 0) st_u32(&h->list_len, len);
+  if (taken == 0 && c.pq_m == 0) {
+    const u32 qid = uld(&h->qid);
+#pragma unroll
+    for (int r = 0; r < NPL; ++r) {
+      const u32 e = (u32)r * 32u + lane;
+      if (e < c.K) write_result(c, qid, e, x[r], e < len);
+    }
+  }
+  return taken;
+}
+
+__device__ u32 merge_select_dispatch(const Ctx &c, u32 qs, u32 lane) {
+  const u32 need = c.L + c.WR;
+  if (need <= 128) return merge_select<4>(c, qs, lane);
+  if (need <= 256) return merge_select<8>(c, qs, lane);
+  return merge_select<16>(c, qs, lane);
+}
+
+// PQ mode: fold the exact distances of the nodes just expanded into the rerank pool
+// (sorted, the best K kept).  Entries K..K+nf-1 of the pool array are the staging area.
+template <int NPL>
+__device__ __noinline__ void pool_merge(const Ctx &c, u32 qs, u32 nf, bool final_out, u32 lane) {
+  QHdr *h = c.hdr + qs;
+  u64 *pool = c.pool + (u64)qs * (c.K + c.W);
+  u32 len = uld(&h->pool_len);
+  u64 x[NPL];
+#pragma unroll
+  for (int r = 0; r < NPL; ++r) {
+    const u32 e = (u32)r * 32u + lane;
+    x[r] = e < len ? ld_u64(pool + e) : (e - len < nf ? ld_u64(pool + c.K + (e - len)) : kPadKey);
+  }
+  if (nf) bitonic_sort<NPL>(x, lane);
+  len = min(c.K, len + nf);
+#pragma unroll
+  for (int r = 0; r < NPL; ++r) {
+    const u32 e = (u32)r * 32u + lane;
+    if (e < len) st_u64(pool + e, x[r]);
+  }
+  if (lane == 0) st_u32(&h->pool_len, len);
+  if (final_out) {
+    const u32 qid = uld(&h->qid);
+#pragma unroll
+    for (int r = 0; r < NPL; ++r) {
+      const u32 e = (u32)r * 32u + lane;
+      if (e < c.K) write_result(c, qid, e, x[r], e < len);
+    }
+  }
+}
+__device__ void pool_merge_dispatch(const Ctx &c, u32 qs, u32 nf, bool final_out, u32 lane) {
+  const u32 need = c.K + c.W;
+  if (need <= 32) pool_merge<1>(c, qs, nf, final_out, lane);
+  else if (need <= 64) pool_merge<2>(c, qs, nf, final_out, lane);
+  else if (need <= 128) pool_merge<4>(c, qs, nf, final_out, lane);
+  else if (need <= 256) pool_merge<8>(c, qs, nf, final_out, lane);
+  else pool_merge<16>(c, qs, nf, final_out, lane);
+}
+
+// Read the adjacency lists delivered by the finished PH_EXPAND batch, drop every neighbour
+// already in the exact visited set, and store the survivors as the next batch's items.
+__device__ u32 collect_neighbors(const Ctx &c, u32 qs, u32 lane) {
+  QHdr *h = c.hdr + qs;
+  const u32 nf = uld(&h->n_items);
+  const u32 *adj = c.adj + (u64)qs * c.W * c.R;
+  const u32 *adjdeg = c.adjdeg + (u64)qs * c.W;
+  u32 *items = c.items + (u64)qs * c.WR;
+  u32 *seen = c.seen + (u64)qs * c.seen_cap;
+  u32 sum_deg = 0;
+  for (u32 f = 0; f < nf; ++f) {
+    u32 d = ld_u32(adjdeg + f);
+    if (d > c.R) { if (lane == 0) raise(c, 7, 0x91, qs, f, d); return 0; }
+    sum_deg += d;
+  }
+  u32 out = 0;
+  const u32 total = nf * c.R;
+  for (u32 base = 0; base < total; base += 32) {
+    const u32 p = base + lane;
+    bool isnew = false;
+    u32 v = 0;
+    if (p < total) {
+      const u32 f = p / c.R, i = p % c.R;
+      if (i < ld_u32(adjdeg + f)) {
+        v = ld_u32(adj + p);
+        if (v >= c.n_nodes) raise(c, 7, 0x92, qs, v);
+        else {
+          u32 r = set_insert(seen, c.seen_cap, v);
+          if (r == 2) raise(c, 6, 0x93, qs, v);
+          isnew = r == 1;
+        }
+      }
+    }
+    const u32 b = __ballot_sync(0xffffffffu, isnew);
+    if (isnew) st_u32(items + out + __popc(b & ((1u << lane) - 1u)), v);
+    out += __popc(b);
+  }
+  __syncwarp();
+  if (lane == 0) {
+    st_u32(&h->sum_deg, ld_u32(&h->sum_deg) + sum_deg);
+    st_u32(&h->n_eval, ld_u32(&h->n_eval) + out);
+  }
+  return out;
+}
+
+// ------------------------------------------------------------------------------------------
+// PQ asymmetric distance: per-query lookup table in shared memory
+// ------------------------------------------------------------------------------------------
+// LUT[m][c] = sum_j (q[m*dsub+j] - cent[m][c][j])^2 (u32, exact); adc(v) = sum_m LUT[m][code[v][m]]
+__device__ void build_lut(const Ctx &c, u32 qid, u32 *lut, u32 lane) {
+  const u8 *q = (const u8 *)c.queries + (u64)qid * c.vec_bytes;
+  const u32 wsub = c.pq_dsub >> 2;
+  const u32 total = c.pq_m * kPqKsub;
+  for (u32 e = lane; e < total; e += 32) {
+    const u32 m = e >> 8;
+    const u32 *cw = (const u32 *)(c.pq_cent + (u64)e * c.pq_dsub);
+    const u32 *qw = (const u32 *)(q + m * c.pq_dsub);
+    u32 s = 0;
+    for (u32 w = 0; w < wsub; ++w) {
+      u32 d = __vabsdiffu4(__ldg(cw + w), __ldg(qw + w));
+      s = __dp4a(d, d, s);
+    }
+    lut[e] = s;
+  }
+  __syncwarp();
+}
+__device__ __forceinline__ u32 warp_adc(const Ctx &c, const u32 *lut, u32 v, u32 lane) {
+  u32 acc = 0;
+  const u8 *code = c.pq_codes + (u64)v * c.pq_m;
+  for (u32 m = lane; m < c.pq_m; m += 32) acc += lut[(m << 8) + __ldg(code + m)];
+  return __reduce_add_sync(0xffffffffu, acc);
+}
+
+// ------------------------------------------------------------------------------------------
+// query life cycle
+// ------------------------------------------------------------------------------------------
+__device__ void finish_query(const Ctx &c, u32 qs, u32 lane) {
+  QHdr *h = c.hdr + qs;
+  if (c.pq_m) pool_merge_dispatch(c, qs, 0, true, lane);
+  __threadfence();
+  __syncwarp();
+  if (lane == 0) {
+    const u32 qid = ld_u32(&h->qid);
+    const u32 pd = ld_u32(&h->pages_distinct), ni = ld_u32(&h->n_iter), nx = ld_u32(&h->n_expand),
+              ne = ld_u32(&h->n_eval), sd = ld_u32(&h->sum_deg);
+    if (c.out_pages) c.out_pages[qid] = pd;
+    if (c.out_counters) {
+      u32 *o = c.out_counters + (u64)qid * 5;
+      o[0] = pd; o[1] = ni; o[2] = nx; o[3] = ne; o[4] = sd;
+    }
+    stat_add(c, S_NEVAL, ne); stat_add(c, S_NEXPAND, nx); stat_add(c, S_SUMDEG, sd);
+    stat_add(c, S_NITER, ni); stat_add(c, S_DONE, 1);
+    __threadfence();
+    u32 d = atomicAdd(&c.ctl->done, 1u) + 1u;
+    if (d == c.nq) st_u32(&c.ctl->stop, 1u);
+  }
+}
+
+__device__ __forceinline__ void reset_hdr(QHdr *h, u32 qid) {
+  st_u32(&h->qid, qid); st_u32(&h->phase, PH_NEW); st_u32(&h->awaiting, 0); st_u32(&h->n_items, 0);
+  st_u32(&h->n_todo, 0); st_u32(&h->list_len, 0); st_u32(&h->n_iter, 0); st_u32(&h->n_expand, 0);
+  st_u32(&h->n_eval, 0); st_u32(&h->sum_deg, 0); st_u32(&h->pages_distinct, 0); st_u32(&h->pool_len, 0);
+}
+
+// The slot's query is done: admit the next unstarted query into the same slot, if any.
+__device__ bool recycle_slot(const Ctx &c, u32 qs, u32 lane) {
+  u32 nxt = 0;
+  if (lane == 0) nxt = atomicAdd(&c.ctl->next_query, 1u);
+  nxt = __shfl_sync(0xffffffffu, nxt, 0);
+  if (nxt >= c.nq) return false;
+  uint4 ff = make_uint4(kInvalidId, kInvalidId, kInvalidId, kInvalidId);
+  uint4 *s4 = (uint4 *)(c.seen + (u64)qs * c.seen_cap);
+  for (u32 i = lane; i < c.seen_cap / 4; i += 32) __stcg(s4 + i, ff);
+  uint4 *p4 = (uint4 *)(c.pset + (u64)qs * c.pset_cap);
+  for (u32 i = lane; i < c.pset_cap / 4; i += 32) __stcg(p4 + i, ff);
+  if (lane == 0) reset_hdr(c.hdr + qs, nxt);
+  __threadfence();
+  __syncwarp();
+  return true;
+}
+
+template <bool PQ>
+__device__ void run_query(const Ctx &c, u32 qs, bool retry, u32 lane, u32 *lut) {
+  QHdr *h = c.hdr + qs;
+  if (retry) {
+    if (!issue_batch(c, qs, true, lane)) return;
+  }
+  for (u32 guard = 0; guard < 4u * c.max_iters + 64u; ++guard) {
+    if (warp_stopped(c)) return;
+    const u32 phase = uld(&h->phase);
+    if (phase == PH_NEW) {
+      const u32 qid = uld(&h->qid);
+      if (lane == 0) {
+        set_insert(c.seen + (u64)qs * c.seen_cap, c.seen_cap, c.entry);
+        st_u32(c.items + (u64)qs * c.WR, c.entry);
+        st_u32(&h->n_items, 1); st_u32(&h->n_eval, 1); st_u32(&h->phase, PH_EVAL);
+      }
+      __syncwarp();
+      if (PQ) {
+        build_lut(c, qid, lut, lane);
+        u32 d = warp_adc(c, lut, c.entry, lane);
+        if (lane == 0) st_u64(c.cand + (u64)qs * c.WR, mk_key(d, c.entry));
+        __syncwarp();
+      } else {
+        if (!issue_batch(c, qs, false, lane)) return;
+      }
+    } else if (phase == PH_EVAL) {
+      const u32 nf = merge_select_dispatch(c, qs, lane);
+      if (nf == 0) {
+        finish_query(c, qs, lane);
+        if (!recycle_slot(c, qs, lane)) return;
+        guard = 0;
+        continue;
+      }
+      if (lane == 0) {
+        const u32 it = ld_u32(&h->n_iter) + 1u;
+        st_u32(&h->n_iter, it); st_u32(&h->n_expand, ld_u32(&h->n_expand) + nf);
+        st_u32(&h->n_items, nf); st_u32(&h->phase, PH_EXPAND);
+        if (it > c.max_iters) raise(c, 6, 0xA1, qs, it);
+      }
+      __syncwarp();
+      if (!issue_batch(c, qs, false, lane)) return;
+    } else {  // PH_EXPAND complete
+      const u32 nf = uld(&h->n_items);
+      const u32 nn = collect_neighbors(c, qs, lane);
+      if (PQ) {
+        pool_merge_dispatch(c, qs, nf, false, lane);
+        const u32 qid = uld(&h->qid);
+        build_lut(c, qid, lut, lane);
+        const u32 *items = c.items + (u64)qs * c.WR;
+        for (u32 i = 0; i < nn; ++i) {
+          const u32 v = ld_u32(items + i);
+          u32 d = warp_adc(c, lut, v, lane);
+          if (lane == 0) st_u64(c.cand + (u64)qs * c.WR + i, mk_key(d, v));
+        }
+      }
+      if (lane == 0) { st_u32(&h->n_items, nn); st_u32(&h->phase, PH_EVAL); }
+      __syncwarp();
+      if (!PQ && nn > 0) {
+        if (!issue_batch(c, qs, false, lane)) return;
+      }
+    }
+  }
+  if (lane == 0) raise(c, 6, 0xA2, qs);
+}
+
+// Warp 0 of block 0: forwards the proxy's completion ring (host memory) into the arrival
+// queue in HBM, watches the host's abort word and the deadline.
+__device__ void poller(const Ctx &c, u32 lane) {
+  u32 seen = 0, it = 0;
+  const u64 t0 = globaltimer();
+  for (;;) {
+    if (warp_stopped(c)) break;
+    u32 tail = 0, abort_req = 0;
+    if (lane == 0) { tail = ld_sys_u32(c.host_ctl); abort_req = ld_sys_u32(c.host_ctl + 1); }
+    tail = __shfl_sync(0xffffffffu, tail, 0);
+    abort_req = __shfl_sync(0xffffffffu, abort_req, 0);
+    if (abort_req) { if (lane == 0) raise(c, 5, 0xB1); break; }
+    while (seen != tail) {
+      const u32 nn = min(32u, tail - seen);
+      if (lane < nn) {
+        u32 slot = ld_sys_u32(c.comp_ring + ((seen + lane) & c.comp_mask));
+        q_push(c, c.arr, slot);
+      }
+      seen += nn;
+      __syncwarp();
+    }
+    u32 late = ((++it & 255u) == 0 && globaltimer() - t0 > c.timeout_ns) ? 1u : 0u;
+    if (__shfl_sync(0xffffffffu, late, 0)) { if (lane == 0) raise(c, 5, 0xB2); break; }
+  }
+}
+
+// Register budget: at most 80 per thread, so that 20 resident warps leave register file and
+// thread slots on every SM for the proxy's copy kernels, which must run concurrently.
+template <bool PQ>
+__global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
+  extern __shared__ u32 smem_lut[];
+  const u32 lane = lane_id(), warp = threadIdx.x >> 5;
+  if (blockIdx.x == 0 && warp == 0) { poller(c, lane); return; }
+  u32 *lut = PQ ? smem_lut + (u64)warp * c.pq_m * kPqKsub : nullptr;
+  const u64 t0 = globaltimer();
+  u32 idle = 0;
+  for (;;) {
+    if (warp_stopped(c)) break;
+    u32 v;
+    if (warp_pop(c, c.arr, v, lane)) { consume_arrival(c, v, lane); idle = 0; continue; }
+    if (warp_pop(c, c.run, v, lane)) { run_query<PQ>(c, v, false, lane, lut); idle = 0; continue; }
+    if (warp_pop(c, c.retry, v, lane)) { run_query<PQ>(c, v, true, lane, lut); idle = 0; __nanosleep(200); continue; }
+    ++idle;
+    __nanosleep(idle < 16 ? 100 : 1000);
+    u32 late = ((idle & 127u) == 0 && globaltimer() - t0 > c.timeout_ns) ? 1u : 0u;
+    if (__shfl_sync(0xffffffffu, late, 0)) { if (lane == 0) raise(c, 5, 0xB3); break; }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// set-up kernels
+// ------------------------------------------------------------------------------------------
+__global__ void init_kernel(const Ctx c) {
+  const u32 tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+  for (u32 i = tid; i < c.n_qslots; i += nth) reset_hdr(c.hdr + i, i);
+  // runnable queue starts with every slot; the others start empty
+  u64 *run = (u64 *)c.run.buf, *arr = (u64 *)c.arr.buf, *rty = (u64 *)c.retry.buf;
+  for (u32 i = tid; i <= c.run.mask; i += nth) run[i] = i < c.n_qslots ? (((u64)(i + 1u) << 32) | i) : ((u64)i << 32);
+  for (u32 i = tid; i <= c.retry.mask; i += nth) rty[i] = (u64)i << 32;
+  for (u32 i = tid; i <= c.arr.mask; i += nth) arr[i] = (u64)i << 32;
+  if (tid == 0) {
+    Ctl *ctl = c.ctl;
+    ctl->stop = 0; ctl->status = 0; ctl->next_query = c.n_qslots; ctl->done = 0; ctl->ring_head = 0;
+    for (int i = 0; i < 8; ++i) { ctl->q_heads[i] = 0; ctl->dbg[i] = 0; }
+    *c.run.tail = c.n_qslots;
+  }
+}
+
+// Empty the cache; slots 0..preloaded-1 are marked READY holding pages 0..preloaded-1
+// (their bytes were copied there by the host before this kernel).
+__global__ void cache_reset_kernel(const Ctx c, u32 preloaded) {
+  const u32 tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+  const u32 n_tags = c.n_sets * kWays;
+  for (u32 ti = tid; ti < n_tags; ti += nth) {
+    const u32 slot = (ti % kWays) * c.n_sets + ti / kWays;
+    const bool pre = slot < preloaded;     // page p preloads into slot p: set p % n_sets, way p / n_sets
+    c.tag[ti] = pre ? mk_tag(slot, 1, 1, ST_READY) : mk_tag(kInvalidId, 0, 0, ST_EMPTY);
+    c.wl[ti] = pre ? ((1ull << 32) | kClosed) : (u64)kClosed;
+  }
+  for (u32 s = tid; s < c.n_sets; s += nth) c.hand[s] = 0;
+}
+
+// Proxy copy batch: block b copies page b of the batch from host-mapped memory into its
+// cache slot (256 threads x 16 bytes); the last block to finish reports the batch sequence
+// number to the host.
+__global__ void fill_kernel(const FillBatch b, const u8 *host_pages, u8 *slot_data, u32 *counter,
+                            u32 *host_copied) {
+  const u32 i = blockIdx.x;
+  const uint4 *src = (const uint4 *)(host_pages + (u64)b.page[i] * kPageBytes);
+  uint4 *dst = (uint4 *)(slot_data + (u64)b.slot[i] * kPageBytes);
+  const uint4 v = __ldcs(src + threadIdx.x);
+  __stcg(dst + threadIdx.x, v);
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    u32 done = atomicAdd(counter, 1u) + 1u;
+    if (done == b.n) {
+      *counter = 0;
+      __threadfence_system();
+      asm volatile("st.relaxed.sys.global.u32 [%0], %1;" ::"l"(host_copied), "r"(b.seq) : "memory");
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// launchers
+// ------------------------------------------------------------------------------------------
+// With lazy module loading the first launch of a kernel may need a context-wide
+// synchronisation, which can never finish while the persistent kernel is waiting for that
+// very launch (the proxy's first copy kernel).  Querying the attributes loads the code now.
+cudaError_t preload_kernels() {
+  cudaFuncAttributes a;
+  cudaError_t e;
+  if ((e = cudaFuncGetAttributes(&a, search_kernel<false>)) != cudaSuccess) return e;
+  if ((e = cudaFuncGetAttributes(&a, search_kernel<true>)) != cudaSuccess) return e;
+  if ((e = cudaFuncGetAttributes(&a, init_kernel)) != cudaSuccess) return e;
+  if ((e = cudaFuncGetAttributes(&a, cache_reset_kernel)) != cudaSuccess) return e;
+  return cudaFuncGetAttributes(&a, fill_kernel);
+}
+
+cudaError_t launch_init(const Ctx &c, cudaStream_t s) {
+  init_kernel<<<148, 256, 0, s>>>(c);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_cache_reset(const Ctx &c, u32 preloaded, cudaStream_t s) {
+  cache_reset_kernel<<<148, 256, 0, s>>>(c, preloaded);
+  return cudaGetLastError();
+}
+
+static size_t search_smem(const Ctx &c, u32 warps) { return c.pq_m ? (size_t)warps * c.pq_m * kPqKsub * 4 : 0; }
+
+cudaError_t search_occupancy(bool pq, u32 warps_per_block, int *blocks_per_sm) {
+  if (pq) return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<true>, warps_per_block * 32,
+                                                               (size_t)warps_per_block * 32 * kPqKsub * 4);
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<false>, warps_per_block * 32, 0);
+}
+
+cudaError_t launch_search(const Ctx &c, u32 blocks, u32 warps_per_block, cudaStream_t s) {
+  const size_t smem = search_smem(c, warps_per_block);
+  if (c.pq_m) {
+    cudaError_t e = cudaFuncSetAttribute(search_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    search_kernel<true><<<blocks, warps_per_block * 32, smem, s>>>(c);
+  } else {
+    search_kernel<false><<<blocks, warps_per_block * 32, 0, s>>>(c);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_fill(const FillBatch &b, const u8 *host_pages_dev, u8 *slot_data, u32 *counter,
+                        u32 *host_copied, cudaStream_t s) {
+  fill_kernel<<<b.n, 256, 0, s>>>(b, host_pages_dev, slot_data, counter, host_copied);
+  return cudaGetLastError();
+}
+
+}  // namespace gorio
