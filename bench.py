@@ -1,0 +1,278 @@
+#!/usr/bin/env python
+"""Benchmark of the GPU-owned paged beam search on the SIFT1M-shaped workload.
+
+One "step" is one blocking search of all 10,000 queries against the 1,000,000-node uint8
+index (R=64, 10 nodes per 4 KB page) starting from a COLD 20 % page cache, with the remote
+tier emulated at 20 us per request and at most 256 requests in service.  The cache is
+re-created (untimed) before every step; an L2 flush precedes every timed region.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+prints one JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "QPS @ recall@10, 1M x 128 uint8, 20% cache, 20us miss"
+PAPER_CONTEXT = ("paper (L40S + ConnectX-6 NVMe-oF, SIFT1M): G-ABaM 5650 QPS = 4.89x over blocking BaM, "
+                 "G-Gust 1.31x over GustANN; context only, other hardware and transport")
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return json.load(open(p)), "measured"
+    return {"hbm_gbs": 6650.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.rows, self.proc, self.gpu = [], None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+        sm = [float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({n for r in self.rows if len(r) >= 7 for n, v in zip(names, r[3:7]) if v == "Active"})
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def measure_h2d_gbs(device):
+    """Pinned host -> device copy bandwidth, 256 MB, best of 10 (the link the page fills cross)."""
+    n = 256 << 20
+    h = torch.empty(n, dtype=torch.uint8).pin_memory()
+    d = torch.empty(n, dtype=torch.uint8, device=device)
+    best = 0.0
+    for _ in range(10):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); d.copy_(h, non_blocking=True); b.record(); torch.cuda.synchronize()
+        best = max(best, n / (a.elapsed_time(b) * 1e-3) / 1e9)
+    return best
+
+
+def l2_flush(buf):
+    buf.add_(1)          # 512 MB read+write, larger than the 126 MB L2
+
+
+def oracle_qps(w, threads, budget_s=20.0):
+    """The CPU oracle as it stands on a bounded sample of the same queries."""
+    from oracle import OracleIndex
+    orc = OracleIndex.from_workload(w)
+    t = time.perf_counter(); orc.search(w.queries[: 4 * threads], w.K, w.L, w.W, threads=threads)
+    per_q = (time.perf_counter() - t) / (4 * threads)
+    n = int(min(w.nq, max(8 * threads, budget_s / max(per_q, 1e-6))))
+    t = time.perf_counter(); orc.search(w.queries[:n], w.K, w.L, w.W, threads=threads)
+    dt = time.perf_counter() - t
+    return n / dt, n
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--scale", type=float, default=1.0, help="shrink the index (profiling captures only)")
+    ap.add_argument("--cache-frac", type=float, default=0.20)
+    ap.add_argument("--preload", action="store_true", help="fully resident cache (profiling captures only)")
+    ap.add_argument("--nq", type=int, default=10_000)
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    threads = os.cpu_count() or 1
+
+    from workloads import make_config, recall_at_k
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        w = make_config(3, scale=args.scale, nq=args.nq, device="cuda" if torch.cuda.is_available() else "cpu",
+                        with_gt=False)
+        vals = []
+        for _ in range(args.warmup):
+            oracle_qps(w, threads, budget_s=2.0)
+        n_s = 0
+        for _ in range(args.steps):
+            v, n_s = oracle_qps(w, threads, budget_s=max(5.0, 60.0 / max(1, args.steps)))
+            vals.append(v)
+        v = statistics.mean(vals)
+        sample = f"first {n_s} of {w.nq} queries per step, {threads} threads, in-memory page store, no cache emulation"
+        print(json.dumps({
+            "impl": "reference", "metric": METRIC, "value": v, "unit": "queries/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * n_s / v, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+            "config": {"workload": f"cfg3 SIFT1M-shaped: N={w.N} d=128 u8 R=64 npp=10 K=10 L=100 W=4"},
+            "cpu_baseline": {"value": v, "unit": "queries/s", "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": v, "unit": "queries/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        }))
+        return
+
+    import paper_2607_04415_b200 as g
+    from paper_2607_04415_b200 import build
+    build.build()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the search has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # every rank searches its own 10,000 queries (weak scaling): query seed 1 + rank
+    w = make_config(3, scale=args.scale, nq=args.nq, device=dev, seed_q=1 + rank)
+    cap = w.n_pages if args.preload else int(args.cache_frac * w.n_pages)
+    lat_ns, max_out = 20_000, 256
+    ix = g.Index.from_workload(w, device=local)
+    q_dev = torch.as_tensor(w.queries).to(dev)
+    q_pin = torch.as_tensor(w.queries).pin_memory()
+    outs_pin = dict(ids=torch.empty((w.nq, w.K), dtype=torch.int32).pin_memory(),
+                    dists=torch.empty((w.nq, w.K), dtype=torch.int32).pin_memory(),
+                    pages=torch.empty(w.nq, dtype=torch.int32).pin_memory(),
+                    counters=torch.empty((w.nq, 5), dtype=torch.int32).pin_memory())
+    flush = torch.zeros(512 << 20, dtype=torch.uint8, device=dev)
+    h2d = measure_h2d_gbs(dev)
+    pk, pk_kind = peaks()
+
+    def reset_cache():
+        ix.cache_config(cap, remote_latency_ns=lat_ns, max_outstanding=max_out, preload=args.preload,
+                        timeout_ms=120_000)
+        ix.stats_reset()
+        l2_flush(flush)
+
+    def one_step():
+        reset_cache()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        out = ix.search(q_dev, w.K, w.L, w.W)
+        b.record()
+        barrier()
+        t = torch.tensor([a.elapsed_time(b)], device=dev)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t), out, ix.stats()
+
+    for _ in range(max(3, args.warmup)):
+        one_step()
+    sampler = ClockSampler(local); sampler.start()
+    times, stats_list, out = [], [], None
+    for _ in range(args.steps):
+        t, out, st = one_step()
+        times.append(t); stats_list.append(st)
+    clocks = sampler.stop()
+
+    # end to end through the host-buffer entry point: H2D queries, search, D2H results
+    e2e_times = []
+    for i in range(1 + min(3, args.steps)):
+        reset_cache()
+        barrier()
+        t0 = time.perf_counter()
+        ix.search_host(q_pin.numpy(), w.K, w.L, w.W, out={k: v.numpy() for k, v in outs_pin.items()})
+        dt = time.perf_counter() - t0
+        tt = torch.tensor([dt], device=dev)
+        if world > 1:
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        if i:
+            e2e_times.append(float(tt))
+    ms = statistics.mean(times)
+    st = stats_list[len(stats_list) // 2]
+    fetched = statistics.mean(s["pages_fetched"] for s in stats_list)
+    launches = sum(2 + s["proxy_batches"] for s in stats_list)
+
+    # roofline: the slowest of (a) algorithmic HBM bytes at the measured copy peak, (b) fetched
+    # page bytes over the measured host link, (c) outstanding window / injected latency
+    b_alg = st["n_eval"] * w.d + 4 * st["n_expand"] + 4 * st["sum_degree"]
+    b_hbm = b_alg + 4096 * fetched
+    t_a = b_hbm / (pk["hbm_gbs"] * 1e9)
+    t_b = 4096 * fetched / (h2d * 1e9)
+    t_c = fetched * lat_ns * 1e-9 / max_out
+    terms = {"hbm": t_a, "host_link": t_b, "outstanding_window": t_c}
+    bound = max(terms, key=terms.get)
+    t_roof = terms[bound]
+    if bound == "hbm":
+        ach, peak, unit = b_hbm / (ms * 1e-3) / 1e9, pk["hbm_gbs"], "GB/s"
+    elif bound == "host_link":
+        ach, peak, unit = 4096 * fetched / (ms * 1e-3) / 1e9, h2d, "GB/s"
+    else:
+        ach, peak, unit = fetched / (ms * 1e-3) / 1e6, max_out / (lat_ns * 1e-9) / 1e6, "Mfetch/s"
+
+    ids = out["ids"].cpu().numpy().view(np.uint32)
+    recall = recall_at_k(ids, w.gt)
+    line = {
+        "metric": METRIC, "value": world * w.nq / (ms * 1e-3), "unit": "queries/s", "n_gpus": world,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": f"cfg3 SIFT1M-shaped: N={w.N} d=128 u8 R=64 npp=10 pages={w.n_pages} "
+                               f"nq={w.nq}/gpu K=10 L=100 W=4 cache={cap} slots cold latency=20us max_outstanding=256",
+                   "recall_at_10": recall, "l2": "flushed before every step (512 MB read+write)",
+                   "cache": "re-created cold before every step, untimed", "parallelism": f"query-sharded x{world}",
+                   "context": PAPER_CONTEXT},
+        "clocks": clocks,
+        "e2e": {"value": world * w.nq / statistics.mean(e2e_times), "unit": "queries/s",
+                "h2d_bytes_per_step": int(q_pin.numel()),
+                "d2h_bytes_per_step": int(sum(v.numel() * 4 for v in outs_pin.values()))},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": t_roof / (ms * 1e-3),
+                     "traffic": None, "peak_kind": f"hbm {pk_kind}; host link measured in this run ({h2d:.1f} GB/s)",
+                     "terms_ms": {k: 1e3 * v for k, v in terms.items()},
+                     "pages_fetched": fetched, "algorithmic_hbm_bytes": b_hbm,
+                     "hbm_achieved_gbs": b_hbm / (ms * 1e-3) / 1e9, "hbm_peak_gbs": pk["hbm_gbs"]},
+        "stats": {k: st[k] for k in ("pages_hit", "pages_missed", "pages_fetched", "dedupe_joins", "evictions",
+                                     "retries", "max_outstanding_seen", "resumes", "proxy_batches")},
+    }
+    if rank == 0 and world == 1:
+        v, n_s = oracle_qps(w, threads)
+        line["cpu_baseline"] = {"value": v, "unit": "queries/s", "cores": threads, "kind": "oracle",
+                                "sample": f"first {n_s} of {w.nq} queries, {threads} threads, in-memory page store "
+                                          "(no cache emulation, no injected latency)"}
+    ix.close()
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -85,9 +85,8 @@ typedef struct {
  *   preload          1: fill the cache with pages 0..capacity-1 now (whole index when
  *                    capacity >= n_pages); 0: start cold.
  *   timeout_ms       bound on one gorio_search call (device and host waits); 0 = 60000.
- *   copy_mode        0: the proxy enqueues batched gather-copy kernels on its own streams;
- *                    1: the proxy issues one cudaMemcpyAsync per page (DMA engine).
- *   fill_batch       pages per proxy copy batch (1..128), 0 = default.
+ *   fill_batch       pages per proxy copy batch (1..128), 0 = default.  The proxy moves
+ *                    pages with batched gather-copy kernels enqueued on its own streams.
  * Calling it again re-creates an empty (or preloaded) cache.
  */
 typedef struct {
@@ -96,8 +95,8 @@ typedef struct {
   uint32_t max_outstanding;
   uint32_t preload;
   uint32_t timeout_ms;
-  uint32_t copy_mode;
   uint32_t fill_batch;
+  uint32_t reserved;
 } gorio_cache_cfg;
 
 /*

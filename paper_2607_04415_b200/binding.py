@@ -37,8 +37,8 @@ class _IndexDesc(ctypes.Structure):
 class _CacheCfg(ctypes.Structure):
     _fields_ = [("capacity_pages", ctypes.c_uint64), ("remote_latency_ns", ctypes.c_uint32),
                 ("max_outstanding", ctypes.c_uint32), ("preload", ctypes.c_uint32),
-                ("timeout_ms", ctypes.c_uint32), ("copy_mode", ctypes.c_uint32),
-                ("fill_batch", ctypes.c_uint32)]
+                ("timeout_ms", ctypes.c_uint32), ("fill_batch", ctypes.c_uint32),
+                ("reserved", ctypes.c_uint32)]
 
 
 class _Tuning(ctypes.Structure):
@@ -128,9 +128,9 @@ class Index:
             raise GorioError(status, detail or self._lib.gorio_status_str(status).decode())
 
     def cache_config(self, capacity_pages, remote_latency_ns=0, max_outstanding=256, preload=False,
-                     timeout_ms=0, copy_mode=0, fill_batch=0):
+                     timeout_ms=0, fill_batch=0):
         cfg = _CacheCfg(int(capacity_pages), int(remote_latency_ns), int(max_outstanding), int(bool(preload)),
-                        int(timeout_ms), int(copy_mode), int(fill_batch))
+                        int(timeout_ms), int(fill_batch), 0)
         self._check(self._lib.gorio_cache_config(self._h, ctypes.byref(cfg)))
 
     def set_tuning(self, max_inflight=0, visited_capacity=0, warps_per_block=0, blocks_per_sm=0):
@@ -152,17 +152,20 @@ class Index:
                                            counters.data_ptr() if want_counters else None, s.cuda_stream))
         return dict(ids=ids, dists=dists, pages_distinct=pages, counters=counters)
 
-    def search_host(self, queries: np.ndarray, K: int, L: int, W: int):
-        """Host buffers in, host buffers out (the copies happen inside the C call)."""
+    def search_host(self, queries: np.ndarray, K: int, L: int, W: int, out: Optional[dict] = None):
+        """Host buffers in, host buffers out (the copies happen inside the C call).  `out` may
+        supply preallocated (e.g. pinned) arrays: ids, dists, pages, counters."""
         q = np.ascontiguousarray(queries)
         nq = q.shape[0]
-        ids = np.empty((nq, K), dtype=np.uint32)
-        dists = np.empty((nq, K), dtype=np.uint32 if self.dtype == "u8" else np.float32)
-        pages = np.empty(nq, dtype=np.uint32)
-        counters = np.empty((nq, 5), dtype=np.uint32)
+        out = out or {}
+        ids = out.get("ids", np.empty((nq, K), dtype=np.uint32))
+        dists = out.get("dists", np.empty((nq, K), dtype=np.uint32 if self.dtype == "u8" else np.float32))
+        pages = out.get("pages", np.empty(nq, dtype=np.uint32))
+        counters = out.get("counters", np.empty((nq, 5), dtype=np.uint32))
         self._check(self._lib.gorio_search_host(self._h, q.ctypes.data, nq, K, L, W, ids.ctypes.data,
                                                 dists.ctypes.data, pages.ctypes.data, counters.ctypes.data))
-        return dict(ids=ids, dists=dists, pages_distinct=pages, counters=counters)
+        return dict(ids=ids.view(np.uint32), dists=dists if self.dtype == "f32" else dists.view(np.uint32),
+                    pages_distinct=pages.view(np.uint32), counters=counters.view(np.uint32))
 
     def stats(self) -> dict:
         s = Stats()

@@ -132,10 +132,6 @@ void free_qstate(gorio_index *ix) {
 // page bytes from pinned host memory into cache slots, and publishes completions no
 // earlier than admission + latency.
 // ---------------------------------------------------------------------------------------
-__global__ void notify_kernel(u32 *host_copied, u32 seq) {
-  asm volatile("st.relaxed.sys.global.u32 [%0], %1;" ::"l"(host_copied), "r"(seq) : "memory");
-}
-
 struct InService { u32 slot; u32 stream; u32 seq; Clock::time_point admitted; };
 
 void proxy_service(gorio_index *ix) {
@@ -174,19 +170,8 @@ void proxy_service(gorio_index *ix) {
       const u32 seq = ++stream_seq[k];
       batch.seq = seq;
       cudaError_t e = cudaSuccess;
-      if (ix->cfg.copy_mode == 0) {
-        e = launch_fill(batch, ix->pages_dev, ix->slot_data, ix->fill_counters + k,
-                        ix->hctl_d + 8 + k, ix->fill_streams[k]);
-      } else {
-        for (u32 i = 0; i < batch.n && e == cudaSuccess; ++i)
-          e = cudaMemcpyAsync(ix->slot_data + (size_t)batch.slot[i] * kPageBytes,
-                              (const u8 *)ix->desc.host_pages + (size_t)batch.page[i] * kPageBytes,
-                              kPageBytes, cudaMemcpyHostToDevice, ix->fill_streams[k]);
-        if (e == cudaSuccess) {
-          notify_kernel<<<1, 1, 0, ix->fill_streams[k]>>>(ix->hctl_d + 8 + k, seq);
-          e = cudaGetLastError();
-        }
-      }
+      e = launch_fill(batch, ix->pages_dev, ix->slot_data, ix->fill_counters + k,
+                      ix->hctl_d + 8 + k, ix->fill_streams[k]);
       if (e != cudaSuccess) { ix->px_error.store(2); return; }
       for (u32 i = 0; i < batch.n; ++i) inflight.push_back({batch.slot[i], (u32)k, seq, now0});
       k = (k + 1) % n_streams;
@@ -279,14 +264,10 @@ int setup_cache(gorio_index *ix) {
   // Warm the whole proxy copy path (kernel code, launch path of every copy stream) before a
   // persistent kernel can depend on it: copy page 0 into slot 0 once per stream.
   {
-    cudaFuncAttributes fa;
-    CK(cudaFuncGetAttributes(&fa, notify_kernel));
     FillBatch wb{};
     wb.n = 1; wb.seq = 0; wb.page[0] = 0; wb.slot[0] = 0;
     for (int i = 0; i < kMaxFillStreams; ++i) {
       CK(launch_fill(wb, ix->pages_dev, ix->slot_data, ix->fill_counters + i, ix->hctl_d + 8 + i, ix->fill_streams[i]));
-      notify_kernel<<<1, 1, 0, ix->fill_streams[i]>>>(ix->hctl_d + 8 + i, 0);
-      CK(cudaGetLastError());
       CK(cudaStreamSynchronize(ix->fill_streams[i]));
     }
   }
@@ -449,9 +430,8 @@ int gorio_index_close(gorio_index *ix) {
 
 int gorio_cache_config(gorio_index *ix, const gorio_cache_cfg *cfg) {
   if (!ix || !cfg) return GORIO_ERR_INVALID_ARG;
-  if (cfg->capacity_pages < kWays || cfg->max_outstanding < 1 || cfg->copy_mode > 1 ||
-      cfg->fill_batch > kMaxFillBatch)
-    return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: capacity >= 16, max_outstanding >= 1, copy_mode 0|1, fill_batch <= 128");
+  if (cfg->capacity_pages < kWays || cfg->max_outstanding < 1 || cfg->fill_batch > kMaxFillBatch)
+    return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: capacity >= 16, max_outstanding >= 1, fill_batch <= 128");
   u64 cap = cfg->capacity_pages < ix->n_pages ? cfg->capacity_pages : ix->n_pages;
   if (cap / kWays * kWays >= (1ull << 24)) return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: at most 2^24 slots");
   CK(cudaSetDevice(ix->dev));
@@ -513,7 +493,7 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   if (pq) { u32 lim = (200u * 1024u) / (d.pq_m * kPqKsub * 4u); if (warps > lim) warps = lim; }
   if (warps < 2) return fail(ix, GORIO_ERR_INVALID_ARG, "search: shared memory cannot hold two PQ tables per block");
   int occ = 0;
-  CK(search_occupancy(pq, warps, &occ));
+  CK(search_occupancy(d.pq_m, warps, &occ));
   if (occ < 1) return fail(ix, GORIO_ERR_INVALID_ARG, "search: launch geometry does not fit an SM");
   u32 bps = ix->tune.blocks_per_sm ? ix->tune.blocks_per_sm : 1u;
   if ((int)bps > occ) bps = (u32)occ;

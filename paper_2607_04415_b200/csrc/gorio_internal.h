@@ -119,7 +119,7 @@ struct FillBatch {
 cudaError_t preload_kernels();
 cudaError_t launch_init(const Ctx &c, cudaStream_t s);
 cudaError_t launch_search(const Ctx &c, u32 blocks, u32 warps_per_block, cudaStream_t s);
-cudaError_t search_occupancy(bool pq, u32 warps_per_block, int *blocks_per_sm);
+cudaError_t search_occupancy(u32 pq_m, u32 warps_per_block, int *blocks_per_sm);
 cudaError_t launch_fill(const FillBatch &b, const u8 *host_pages_dev, u8 *slot_data,
                         u32 *counter, u32 *host_copied, cudaStream_t s);
 cudaError_t launch_cache_reset(const Ctx &c, u32 preloaded_pages, cudaStream_t s);

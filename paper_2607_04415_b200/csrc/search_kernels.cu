@@ -955,9 +955,13 @@ cudaError_t launch_cache_reset(const Ctx &c, u32 preloaded, cudaStream_t s) {
 
 static size_t search_smem(const Ctx &c, u32 warps) { return c.pq_m ? (size_t)warps * c.pq_m * kPqKsub * 4 : 0; }
 
-cudaError_t search_occupancy(bool pq, u32 warps_per_block, int *blocks_per_sm) {
-  if (pq) return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<true>, warps_per_block * 32,
-                                                               (size_t)warps_per_block * 32 * kPqKsub * 4);
+cudaError_t search_occupancy(u32 pq_m, u32 warps_per_block, int *blocks_per_sm) {
+  if (pq_m) {
+    const size_t smem = (size_t)warps_per_block * pq_m * kPqKsub * 4;
+    cudaError_t e = cudaFuncSetAttribute(search_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<true>, warps_per_block * 32, smem);
+  }
   return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<false>, warps_per_block * 32, 0);
 }
 

@@ -1,0 +1,338 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, element by
+element on the same seeded inputs.  uint8 data must match bit-exactly (ids, integer
+distances, per-query counters); fp32 within the tolerance procedure below."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import OracleIndex
+from workloads import make_config, make_workload, recall_at_k, train_pq, write_page_store
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gorio():
+    from paper_2607_04415_b200 import build
+    build.build()
+    import paper_2607_04415_b200 as g
+    return g
+
+
+def _u32(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+def _gpu_search(g, w, capacity, L=None, W=None, K=None, use_pq=False, queries=None, tuning=None, **cfg):
+    ix = g.Index.from_workload(w, use_pq=use_pq)
+    try:
+        cfg.setdefault("timeout_ms", 60000)
+        ix.cache_config(capacity, **cfg)
+        if tuning:
+            ix.set_tuning(**tuning)
+        q = torch.as_tensor(w.queries if queries is None else queries).cuda()
+        out = ix.search(q, K or w.K, L or w.L, W or w.W)
+        torch.cuda.synchronize()
+        res = dict(ids=_u32(out["ids"]), counters=_u32(out["counters"]), pages=_u32(out["pages_distinct"]),
+                   dists=_u32(out["dists"]) if w.dtype == "u8" else out["dists"].cpu().numpy(),
+                   stats=ix.stats())
+        return res
+    finally:
+        ix.close()
+
+
+def _assert_exact(got, ref, rows=None):
+    sl = slice(None) if rows is None else rows
+    assert (got["ids"][sl] == ref["ids"][sl]).all()
+    assert (got["dists"][sl] == ref["dists"][sl]).all()
+    assert (got["counters"][sl] == ref["counters"][sl]).all()
+    assert (got["pages"][sl] == ref["counters"][sl][:, 0]).all()
+
+
+def _check_stats_invariants(st, ref_counters, max_outstanding, union_pages=None, preloaded=0):
+    assert st["pages_fetched"] <= st["pages_missed"]
+    assert int(ref_counters[:, 0].sum()) <= st["pages_hit"] + st["pages_missed"]
+    assert st["max_outstanding_seen"] <= max_outstanding
+    assert st["queries_done"] == ref_counters.shape[0]
+    assert st["n_eval"] == int(ref_counters[:, 3].sum())
+    assert st["n_expand"] == int(ref_counters[:, 2].sum())
+    assert st["sum_degree"] == int(ref_counters[:, 4].sum())
+    if union_pages is not None:
+        assert st["pages_fetched"] >= union_pages - preloaded
+
+
+# ------------------------------------------------------------------ configs 1 and 2 (10k nodes)
+@pytest.fixture(scope="module")
+def cfg1():
+    w = make_config(1)
+    ref = OracleIndex.from_workload(w).search(w.queries, w.K, w.L, w.W, threads=8, want_union=True)
+    return w, ref
+
+
+def test_config1_fully_cached_bit_exact(gorio, cfg1):
+    w, ref = cfg1
+    got = _gpu_search(gorio, w, w.n_pages, preload=True)
+    _assert_exact(got, ref)
+    st = got["stats"]
+    assert st["pages_missed"] == 0 and st["pages_fetched"] == 0       # whole index resident
+    _check_stats_invariants(st, ref["counters"], 256)
+    assert recall_at_k(got["ids"], w.gt) == recall_at_k(ref["ids"], w.gt)
+
+
+def test_config2_ten_percent_cache_bit_exact(gorio, cfg1):
+    w, ref = cfg1
+    cap = int(0.10 * w.n_pages)
+    got = _gpu_search(gorio, w, cap, remote_latency_ns=0, max_outstanding=256)
+    _assert_exact(got, ref)
+    st = got["stats"]
+    assert st["pages_missed"] > 0 and st["dedupe_joins"] > 0 and st["evictions"] > 0 and st["resumes"] > 0
+    _check_stats_invariants(st, ref["counters"], 256, union_pages=int(ref["page_union"].sum()))
+
+
+def test_cold_cache_with_room_for_every_page_fetches_each_page_once(gorio, cfg1):
+    """Dedupe proof: with capacity for every page nothing is evicted, so the number of
+    descriptors serviced must equal the number of distinct pages all queries touched."""
+    w, ref = cfg1
+    got = _gpu_search(gorio, w, w.n_pages, preload=False, max_outstanding=256)
+    _assert_exact(got, ref)
+    assert got["stats"]["pages_fetched"] == int(ref["page_union"].sum())
+    assert got["stats"]["evictions"] == 0
+
+
+@pytest.mark.parametrize("cfg", [
+    dict(capacity=16), dict(capacity=64, max_outstanding=1), dict(capacity=1000, remote_latency_ns=20000),
+    dict(capacity=1000, remote_latency_ns=200000, max_outstanding=32),
+    dict(capacity=1000, fill_batch=1), dict(capacity=1000, fill_batch=128, max_outstanding=1024),
+    dict(capacity=2500, tuning=dict(warps_per_block=4)), dict(capacity=2500, tuning=dict(max_inflight=48)),
+    dict(capacity=2500, tuning=dict(warps_per_block=8, blocks_per_sm=2)),
+], ids=lambda c: "-".join(f"{k}={v}" for k, v in c.items() if k != "tuning") + ("-tuned" if "tuning" in c else ""))
+def test_results_do_not_depend_on_cache_proxy_or_geometry(gorio, cfg1, cfg):
+    """The proxy never touches search state, so outputs must be identical under any cache
+    size, latency, outstanding depth, batch size and launch geometry."""
+    w, ref = cfg1
+    cfg = dict(cfg)
+    cap = cfg.pop("capacity")
+    nq = 200 if cap < 100 else 1000
+    got = _gpu_search(gorio, w, cap, queries=w.queries[:nq], **cfg)
+    _assert_exact(got, ref, rows=slice(0, nq))
+    assert got["stats"]["max_outstanding_seen"] <= cfg.get("max_outstanding", 256)
+
+
+def test_host_buffer_entry_point_matches(gorio, cfg1):
+    w, ref = cfg1
+    ix = gorio.Index.from_workload(w)
+    try:
+        ix.cache_config(2000, remote_latency_ns=5000)
+        out = ix.search_host(w.queries, w.K, w.L, w.W)
+    finally:
+        ix.close()
+    assert (out["ids"] == ref["ids"]).all() and (out["dists"] == ref["dists"]).all()
+    assert (out["counters"] == ref["counters"]).all() and (out["pages_distinct"] == ref["counters"][:, 0]).all()
+
+
+@pytest.mark.parametrize("K,L,W", [(1, 1, 1), (10, 10, 1), (64, 64, 4), (10, 200, 8), (100, 256, 16), (5, 33, 3)])
+def test_parameter_edges(gorio, cfg1, K, L, W):
+    w, _ = cfg1
+    q = w.queries[:64]
+    ref = OracleIndex.from_workload(w).search(q, K, L, W)
+    got = _gpu_search(gorio, w, 1500, K=K, L=L, W=W, queries=q)
+    _assert_exact(got, ref)
+
+
+def test_single_query_and_unreachable_results_are_padded(gorio):
+    from helpers import ring_index
+    data, deg, nbrs, pages = ring_index([0, 10, 20, 30, 40], d=4, npp=2)
+    deg[:] = 0
+    pages = write_page_store(data, deg, nbrs, 2)
+    ix = gorio.Index(pages, 5, 4, "u8", 2, 2, 1)
+    try:
+        ix.cache_config(16)
+        out = ix.search(torch.zeros((1, 4), dtype=torch.uint8).cuda(), 3, 4, 2)
+        assert _u32(out["ids"]).tolist() == [[1, 0xFFFFFFFF, 0xFFFFFFFF]]
+        assert _u32(out["dists"]).tolist() == [[100, 0xFFFFFFFF, 0xFFFFFFFF]]
+        assert _u32(out["counters"]).tolist() == [[1, 1, 1, 1, 0]]
+    finally:
+        ix.close()
+
+
+def test_ring_worked_example_on_gpu(gorio):
+    from helpers import ring_index
+    data, deg, nbrs, pages = ring_index([10 * i for i in range(8)], d=4, npp=2)
+    ix = gorio.Index(pages, 8, 4, "u8", 2, 2, 3)
+    try:
+        ix.cache_config(16)
+        q = torch.tensor([[62, 0, 0, 0]], dtype=torch.uint8).cuda()
+        out = ix.search(q, 2, 3, 2)
+        assert _u32(out["ids"]).tolist() == [[6, 7]] and _u32(out["dists"]).tolist() == [[4, 64]]
+        assert _u32(out["counters"]).tolist() == [[4, 5, 6, 8, 12]]
+    finally:
+        ix.close()
+
+
+# ------------------------------------------------------------------ failure handling without faults
+def test_corrupt_page_is_reported_not_trapped(gorio):
+    from helpers import ring_index
+    data, deg, nbrs, pages = ring_index([0, 10, 20, 30], d=4, npp=1)
+    nbrs[0, 0] = 1234                                    # neighbour id >= N
+    pages = write_page_store(data, deg, nbrs, 1)
+    ix = gorio.Index(pages, 4, 4, "u8", 2, 1, 0)
+    try:
+        ix.cache_config(16)
+        with pytest.raises(gorio.GorioError) as e:
+            ix.search(torch.zeros((2, 4), dtype=torch.uint8).cuda(), 1, 4, 1)
+        assert e.value.status == 7
+    finally:
+        ix.close()
+
+
+def test_visited_set_overflow_is_a_capacity_error_and_index_stays_usable(gorio, cfg1):
+    w, ref = cfg1
+    ix = gorio.Index.from_workload(w)
+    try:
+        ix.cache_config(w.n_pages, preload=True)
+        ix.set_tuning(visited_capacity=256)               # far fewer than the ~1000 nodes a query scores
+        q = torch.as_tensor(w.queries[:32]).cuda()
+        with pytest.raises(gorio.GorioError) as e:
+            ix.search(q, w.K, w.L, w.W)
+        assert e.value.status == 6
+        ix.set_tuning()                                   # defaults again: same index, same context
+        out = ix.search(q, w.K, w.L, w.W)
+        assert (_u32(out["ids"]) == ref["ids"][:32]).all()
+    finally:
+        ix.close()
+
+
+def test_remote_tier_that_never_answers_times_out_cleanly(gorio, cfg1):
+    """The wait runs out (completions are held back by a 4 s latency against a 300 ms
+    budget): the search returns TIMEOUT, every kernel has exited, and the same index then
+    searches correctly again."""
+    w, ref = cfg1
+    ix = gorio.Index.from_workload(w)
+    try:
+        ix.cache_config(1000, remote_latency_ns=4_000_000_000, timeout_ms=300)
+        q = torch.as_tensor(w.queries[:100]).cuda()
+        with pytest.raises(gorio.GorioError) as e:
+            ix.search(q, w.K, w.L, w.W)
+        assert e.value.status == 5
+        ix.cache_config(1000, remote_latency_ns=0, timeout_ms=60000)
+        out = ix.search(q, w.K, w.L, w.W)
+        assert (_u32(out["ids"]) == ref["ids"][:100]).all()
+    finally:
+        ix.close()
+
+
+def test_call_order_and_argument_checks(gorio, cfg1):
+    w, _ = cfg1
+    ix = gorio.Index.from_workload(w)
+    try:
+        q = torch.as_tensor(w.queries[:4]).cuda()
+        with pytest.raises(gorio.GorioError) as e:
+            ix.search(q, 10, 64, 4)                        # before cache_config
+        assert e.value.status == 4
+        ix.cache_config(64)
+        for K, L, W in ((0, 8, 1), (9, 8, 1), (1, 257, 1), (1, 8, 0), (1, 8, 17)):
+            with pytest.raises(gorio.GorioError) as e:
+                ix.search(q, K, L, W)
+            assert e.value.status == 1
+        with pytest.raises(gorio.GorioError):
+            ix.cache_config(8)                             # below one set
+    finally:
+        ix.close()
+
+
+# ------------------------------------------------------------------ config 3 (SIFT1M-shaped)
+def test_config3_scaled_with_latency_bit_exact(gorio):
+    w = make_config(3, scale=0.05, nq=1500)
+    ref = OracleIndex.from_workload(w).search(w.queries, w.K, w.L, w.W, threads=8, want_union=True)
+    got = _gpu_search(gorio, w, w.cache_pages, remote_latency_ns=20000, max_outstanding=256)
+    _assert_exact(got, ref)
+    _check_stats_invariants(got["stats"], ref["counters"], 256, union_pages=int(ref["page_union"].sum()))
+
+
+@pytest.fixture(scope="module")
+def cfg3_full():
+    return make_config(3)
+
+
+def test_config3_full_size_sampled_bit_exact(gorio, cfg3_full):
+    """1M nodes, 10,000 queries, 20% cache, 20 us, <=256 outstanding -- the configuration the
+    benchmark times; the oracle checks a sample of the outputs one by one."""
+    w = cfg3_full
+    assert w.N == 1_000_000 and w.n_pages == 100_000 and w.node_bytes == 388
+    sample = np.arange(0, w.nq, 40)
+    orc = OracleIndex.from_workload(w)
+    ref = orc.search(w.queries[sample], w.K, w.L, w.W, threads=8)
+    got = _gpu_search(gorio, w, w.cache_pages, remote_latency_ns=20000, max_outstanding=256)
+    for key in ("ids", "dists", "counters"):
+        assert (got[key][sample] == ref[key]).all()
+    st = got["stats"]
+    assert st["queries_done"] == w.nq and st["max_outstanding_seen"] <= 256
+    assert st["pages_fetched"] <= st["pages_missed"]
+    # properties that hold at any size: sorted unique output, distances recomputable
+    ids, dd = got["ids"], got["dists"]
+    keys = dd.astype(np.uint64) << np.uint64(32) | ids.astype(np.uint64)
+    assert (keys[:, 1:] > keys[:, :-1]).all()
+    rows = np.arange(0, w.nq, 97)
+    for r in rows:
+        diff = w.data[ids[r]].astype(np.int64) - w.queries[r].astype(np.int64)
+        assert ((diff * diff).sum(1) == dd[r]).all()
+    assert recall_at_k(ids[sample], w.gt[sample]) == recall_at_k(ref["ids"], w.gt[sample])
+
+
+# ------------------------------------------------------------------ config 4 (PQ navigation)
+@pytest.fixture(scope="module")
+def cfg4_small():
+    w = make_config(3, scale=0.05, nq=300)
+    w.pq_centroids, w.pq_codes = train_pq(w.data, m=32, sample=16384, iters=6)
+    return w
+
+
+@pytest.mark.parametrize("L", [50, 100, 200])
+@pytest.mark.parametrize("W", [1, 4, 8])
+def test_config4_pq_sweep_bit_exact(gorio, cfg4_small, L, W):
+    w = cfg4_small
+    ref = OracleIndex.from_workload(w, use_pq=True).search(w.queries, w.K, L, W, threads=8)
+    for frac, preload in ((0.05, False), (0.20, False), (1.0, True)):
+        cap = max(16, int(frac * w.n_pages))
+        got = _gpu_search(gorio, w, cap, L=L, W=W, use_pq=True, preload=preload,
+                          remote_latency_ns=20000 if not preload else 0)
+        _assert_exact(got, ref)
+
+
+def test_config4_full_size_sampled_bit_exact(gorio, cfg3_full):
+    w = cfg3_full
+    if w.pq_centroids is None:
+        w.pq_centroids, w.pq_codes = train_pq(w.data, m=32)
+    sample = np.arange(0, w.nq, 50)
+    ref = OracleIndex.from_workload(w, use_pq=True).search(w.queries[sample], w.K, 100, 4, threads=8)
+    got = _gpu_search(gorio, w, w.cache_pages, L=100, W=4, use_pq=True, remote_latency_ns=20000)
+    for key in ("ids", "dists", "counters"):
+        assert (got[key][sample] == ref[key]).all()
+
+
+# ------------------------------------------------------------------ config 5 (fp32)
+def _fp32_parity(w, got, ref, rows=None):
+    """>= 99.9 % of queries have identical ids; every other query must differ only by swaps
+    or substitutions among near ties (true distances within 1e-5 relative, rank by rank);
+    recall@10 within 0.001; counters identical wherever the ids are."""
+    rows = np.arange(w.nq) if rows is None else rows
+    gi, ri = got["ids"][rows], ref["ids"]
+    same = (gi == ri).all(1)
+    assert same.mean() >= 0.999, f"id match rate {same.mean():.5f}"
+    q64 = w.queries[rows].astype(np.float64)
+    for r in np.nonzero(~same)[0]:
+        assert len(set(gi[r].tolist())) == gi.shape[1]
+        dg = ((w.data[gi[r]].astype(np.float64) - q64[r]) ** 2).sum(1)
+        do = ((w.data[ri[r]].astype(np.float64) - q64[r]) ** 2).sum(1)
+        assert (np.abs(dg - do) <= 1e-5 * do).all(), f"query {rows[r]}: unexplained mismatch"
+        assert (dg[1:] >= dg[:-1] * (1 - 1e-5)).all()
+    np.testing.assert_allclose(got["dists"][rows][same], ref["dists"][same], rtol=2e-6)
+    assert (got["counters"][rows][same] == ref["counters"][same]).mean() >= 0.999
+    assert abs(recall_at_k(gi, w.gt[rows]) - recall_at_k(ri, w.gt[rows])) <= 0.001
+
+
+def test_config5_scaled_fp32_tolerance(gorio):
+    w = make_config(5, scale=0.02, nq=2000)          # 200,000 nodes, 6 per page, 10% cache
+    ref = OracleIndex.from_workload(w).search(w.queries, w.K, w.L, w.W, threads=8)
+    got = _gpu_search(gorio, w, w.cache_pages, remote_latency_ns=20000, max_outstanding=256)
+    _fp32_parity(w, got, ref)

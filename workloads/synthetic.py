@@ -396,12 +396,12 @@ class Workload:
 
 
 def make_workload(name, kind, N, C, nq, d, k, n_rand, npp, clustered_knn, cross_only,
-                  with_pq=False, with_gt=True, device=None, **search):
+                  with_pq=False, with_gt=True, device=None, seed_q=1, **search):
     """Generate vectors, graph, page store (and optionally PQ and ground truth)."""
     if kind == "u8":
-        data, assign, queries = gen_u8(N, C, nq, d)
+        data, assign, queries = gen_u8(N, C, nq, d, seed_q=seed_q)
     else:
-        data, assign, queries = gen_f32(N, C, nq, d)
+        data, assign, queries = gen_f32(N, C, nq, d, seed_q=seed_q)
     deg, nbrs = knn_graph(data, k, n_rand, groups=assign if clustered_knn else None,
                           seed=2, cross_only=cross_only, device=device)
     entry = medoid(data)
@@ -415,14 +415,14 @@ def make_workload(name, kind, N, C, nq, d, k, n_rand, npp, clustered_knn, cross_
     return w
 
 
-def make_config(index, scale=1.0, nq=None, device=None, with_gt=True):
+def make_config(index, scale=1.0, nq=None, device=None, with_gt=True, seed_q=1):
     """The five evaluation configurations (1-based index). ``scale`` < 1 shrinks N and the
     cluster count together so cluster sizes, degrees and page packing keep their shape."""
     def sc(x, lo=1):
         return max(lo, int(round(x * scale)))
     if index in (1, 2):
         w = make_workload(f"cfg{index}", "u8", sc(10_000, 64), 16, nq or 1000, 128, 24, 8, 1,
-                          clustered_knn=False, cross_only=False, device=device, with_gt=with_gt,
+                          clustered_knn=False, cross_only=False, device=device, with_gt=with_gt, seed_q=seed_q,
                           K=10, L=64, W=4)
         if index == 1:
             w.cache_frac, w.preload, w.latency_us = 1.0, True, 0.0
@@ -432,13 +432,13 @@ def make_config(index, scale=1.0, nq=None, device=None, with_gt=True):
     if index in (3, 4):
         w = make_workload(f"cfg{index}", "u8", sc(1_000_000, 4096), sc(256, 2), nq or 10_000, 128,
                           48, 16, 10, clustered_knn=True, cross_only=True, with_pq=(index == 4),
-                          device=device, with_gt=with_gt, K=10, L=100, W=4)
+                          device=device, with_gt=with_gt, seed_q=seed_q, K=10, L=100, W=4)
         w.cache_frac, w.preload, w.latency_us, w.max_outstanding = 0.20, False, 20.0, 256
         return w
     if index == 5:
         w = make_workload("cfg5", "f32", sc(10_000_000, 4096), sc(4096, 2), nq or 10_000, 96,
                           48, 16, 6, clustered_knn=True, cross_only=False, device=device,
-                          with_gt=with_gt, K=10, L=128, W=4)
+                          with_gt=with_gt, seed_q=seed_q, K=10, L=128, W=4)
         w.cache_frac, w.preload, w.latency_us, w.max_outstanding = 0.10, False, 20.0, 256
         return w
     raise ValueError("config index must be 1..5")
