@@ -42,16 +42,18 @@ struct gorio_index {
   // cache
   gorio_cache_cfg cfg{};
   bool cache_ready = false, cache_dirty = false;
-  u32 n_sets = 0, n_slots = 0, preloaded = 0;
+  u32 n_slots = 0, preloaded = 0;
   u8 *slot_data = nullptr;
-  u64 *tag = nullptr, *wl = nullptr;
-  u32 *hand = nullptr;
+  u64 *ptab = nullptr, *smeta = nullptr;
+  u32 *parts = nullptr;
+  CacheShared *cs = nullptr;
+  u64 *want_buf = nullptr; u32 want_cap = 0;
   // host-mapped communication areas
   u64 *ring_h = nullptr; u64 *ring_d = nullptr; u32 ring_cap = 0;
   u32 *comp_h = nullptr; u32 *comp_d = nullptr;
   u32 *hctl_h = nullptr; u32 *hctl_d = nullptr;     // [0] completion tail, [1] abort, [8..] copied flags
   u32 *fill_counters = nullptr;                     // device, one per fill stream
-  u64 *arr_buf = nullptr;
+  u64 *arr_buf = nullptr; u32 arr_cap = 0;
 
   // query state
   gorio_tuning tune{};
@@ -59,7 +61,7 @@ struct gorio_index {
   void *qs_block = nullptr;
   Ctx ctx{};
   Ctl *ctl = nullptr;
-  u64 *run_buf = nullptr, *retry_buf = nullptr; u32 runq_cap = 0;
+  u64 *run_buf = nullptr; u32 runq_cap = 0;
 
   // host-buffer search staging
   void *st_q = nullptr; size_t st_q_bytes = 0;
@@ -113,18 +115,19 @@ cudaError_t host_mapped(T **h, T **d, size_t count) {
 }
 
 void free_cache(gorio_index *ix) {
-  cudaFree(ix->slot_data); cudaFree(ix->tag); cudaFree(ix->wl); cudaFree(ix->hand);
-  cudaFree(ix->arr_buf); cudaFree(ix->fill_counters);
+  cudaFree(ix->slot_data); cudaFree(ix->ptab); cudaFree(ix->smeta); cudaFree(ix->parts); cudaFree(ix->cs);
+  cudaFree(ix->want_buf); cudaFree(ix->fill_counters);
   if (ix->ring_h) cudaFreeHost(ix->ring_h);
   if (ix->comp_h) cudaFreeHost(ix->comp_h);
-  ix->slot_data = nullptr; ix->tag = ix->wl = nullptr; ix->hand = nullptr; ix->arr_buf = nullptr;
+  ix->slot_data = nullptr; ix->ptab = ix->smeta = nullptr; ix->parts = nullptr; ix->cs = nullptr;
+  ix->want_buf = nullptr;
   ix->fill_counters = nullptr; ix->ring_h = ix->ring_d = nullptr; ix->comp_h = ix->comp_d = nullptr;
   ix->cache_ready = false;
 }
 
 void free_qstate(gorio_index *ix) {
-  cudaFree(ix->qs_block); cudaFree(ix->run_buf); cudaFree(ix->retry_buf);
-  ix->qs_block = nullptr; ix->run_buf = ix->retry_buf = nullptr; ix->qs_slots = 0;
+  cudaFree(ix->qs_block); cudaFree(ix->run_buf); cudaFree(ix->arr_buf);
+  ix->qs_block = nullptr; ix->run_buf = ix->arr_buf = nullptr; ix->qs_slots = 0;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -248,15 +251,16 @@ int setup_cache(gorio_index *ix) {
   const gorio_cache_cfg &cfg = ix->cfg;
   free_cache(ix);
   const u64 cap = cfg.capacity_pages;
-  if (cap >= ix->n_pages) ix->n_sets = (ix->n_pages + kWays - 1) / kWays;
-  else ix->n_sets = (u32)(cap / kWays);
-  ix->n_slots = ix->n_sets * kWays;
+  ix->n_slots = cap >= ix->n_pages ? ix->n_pages : (u32)cap;
   ix->ring_cap = next_pow2(2ull * ix->n_slots < 1024 ? 1024 : 2ull * ix->n_slots);
+  ix->want_cap = next_pow2(ix->n_pages < 64 ? 64 : ix->n_pages);
+  free_qstate(ix);               // the arrival queue is sized from the slot count
   CK(cudaMalloc(&ix->slot_data, (size_t)ix->n_slots * kPageBytes));
-  CK(cudaMalloc(&ix->tag, (size_t)ix->n_slots * 8));
-  CK(cudaMalloc(&ix->wl, (size_t)ix->n_slots * 8));
-  CK(cudaMalloc(&ix->hand, (size_t)ix->n_sets * 4));
-  CK(cudaMalloc(&ix->arr_buf, (size_t)ix->ring_cap * 8));
+  CK(cudaMalloc(&ix->ptab, (size_t)ix->n_pages * 8));
+  CK(cudaMalloc(&ix->smeta, (size_t)ix->n_slots * 8));
+  CK(cudaMalloc(&ix->parts, (size_t)ix->n_slots * 4));
+  CK(cudaMalloc(&ix->cs, sizeof(CacheShared)));
+  CK(cudaMalloc(&ix->want_buf, (size_t)ix->want_cap * 8));
   CK(cudaMalloc(&ix->fill_counters, kMaxFillStreams * 4));
   CK(cudaMemset(ix->fill_counters, 0, kMaxFillStreams * 4));
   CK(host_mapped(&ix->ring_h, &ix->ring_d, ix->ring_cap));
@@ -277,7 +281,8 @@ int setup_cache(gorio_index *ix) {
     CK(cudaMemcpy(ix->slot_data, ix->desc.host_pages, (size_t)ix->preloaded * kPageBytes, cudaMemcpyHostToDevice));
   }
   Ctx c{};
-  c.tag = ix->tag; c.wl = ix->wl; c.hand = ix->hand; c.n_sets = ix->n_sets; c.n_slots = ix->n_slots;
+  c.ptab = ix->ptab; c.smeta = ix->smeta; c.parts = ix->parts; c.cs = ix->cs;
+  c.n_slots = ix->n_slots; c.n_pages = ix->n_pages;
   CK(launch_cache_reset(c, ix->preloaded, ix->own_stream));
   CK(cudaStreamSynchronize(ix->own_stream));
   ix->cache_ready = true;
@@ -306,19 +311,19 @@ int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W) {
   const size_t o_wrec = off; off += al((size_t)slots * WR * 4);
   const size_t o_adj = off;  off += al((size_t)slots * WR * 4);
   const size_t o_adeg = off; off += al((size_t)slots * W * 4);
-  const size_t o_todo = off; off += al((size_t)slots * WR * 2);
   const size_t o_pool = off; off += al((size_t)slots * (K + W) * 8);
   const size_t o_seen = off; off += al((size_t)slots * seen_cap * 4);
   const size_t o_pset = off; off += al((size_t)slots * pset_cap * 4);
   CK(cudaMalloc(&ix->qs_block, off));
   ix->runq_cap = next_pow2(2ull * slots < 64 ? 64 : 2ull * slots);
   CK(cudaMalloc(&ix->run_buf, (size_t)ix->runq_cap * 8));
-  CK(cudaMalloc(&ix->retry_buf, (size_t)ix->runq_cap * 8));
+  ix->arr_cap = next_pow2(2ull * ix->n_slots + (u64)slots * WR / 32 + 1024);
+  CK(cudaMalloc(&ix->arr_buf, (size_t)ix->arr_cap * 8));
   u8 *b = (u8 *)ix->qs_block;
   Ctx &c = ix->ctx;
   c.hdr = (QHdr *)(b + o_hdr); c.list = (u64 *)(b + o_list); c.cand = (u64 *)(b + o_cand);
   c.items = (u32 *)(b + o_items); c.wrec = (u32 *)(b + o_wrec); c.adj = (u32 *)(b + o_adj);
-  c.adjdeg = (u32 *)(b + o_adeg); c.todo = (u16 *)(b + o_todo); c.pool = (u64 *)(b + o_pool);
+  c.adjdeg = (u32 *)(b + o_adeg); c.pool = (u64 *)(b + o_pool);
   c.seen = (u32 *)(b + o_seen); c.pset = (u32 *)(b + o_pset);
   c.seen_cap = seen_cap; c.pset_cap = pset_cap; c.n_qslots = slots;
   ix->qs_slots = slots; ix->qs_L = L; ix->qs_W = W; ix->qs_WR = WR; ix->qs_K = K;
@@ -430,14 +435,14 @@ int gorio_index_close(gorio_index *ix) {
 
 int gorio_cache_config(gorio_index *ix, const gorio_cache_cfg *cfg) {
   if (!ix || !cfg) return GORIO_ERR_INVALID_ARG;
-  if (cfg->capacity_pages < kWays || cfg->max_outstanding < 1 || cfg->fill_batch > kMaxFillBatch)
+  if (cfg->capacity_pages < 16 || cfg->max_outstanding < 1 || cfg->fill_batch > kMaxFillBatch)
     return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: capacity >= 16, max_outstanding >= 1, fill_batch <= 128");
   u64 cap = cfg->capacity_pages < ix->n_pages ? cfg->capacity_pages : ix->n_pages;
-  if (cap / kWays * kWays >= (1ull << 24)) return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: at most 2^24 slots");
+  if (cap >= (1ull << 24)) return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: at most 2^24 slots");
   CK(cudaSetDevice(ix->dev));
   ix->cfg = *cfg;
   if (ix->cfg.timeout_ms == 0) ix->cfg.timeout_ms = 60000;
-  if (ix->cfg.fill_batch == 0) ix->cfg.fill_batch = 64;
+  if (ix->cfg.fill_batch == 0) ix->cfg.fill_batch = 128;
   return setup_cache(ix);
 }
 
@@ -473,14 +478,15 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   c.n_nodes = (u32)d.n_nodes; c.dim = d.dim; c.dtype = d.dtype; c.R = d.max_degree; c.npp = d.nodes_per_page;
   c.node_bytes = ix->node_bytes; c.vec_bytes = ix->vec_bytes; c.entry = d.entry_id; c.n_pages = ix->n_pages;
   c.pq_m = d.pq_m; c.pq_dsub = d.pq_m ? d.dim / d.pq_m : 0; c.pq_cent = d.pq_centroids_dev; c.pq_codes = d.pq_codes_dev;
-  c.slot_data = ix->slot_data; c.tag = ix->tag; c.wl = ix->wl; c.hand = ix->hand;
-  c.n_sets = ix->n_sets; c.n_slots = ix->n_slots;
+  c.slot_data = ix->slot_data; c.ptab = ix->ptab; c.smeta = ix->smeta; c.parts = ix->parts; c.cs = ix->cs;
+  c.n_slots = ix->n_slots;
   c.ring = ix->ring_d; c.ring_mask = ix->ring_cap - 1; c.ring_shift = ilog2(ix->ring_cap);
   c.comp_ring = ix->comp_d; c.comp_mask = ix->ring_cap - 1; c.host_ctl = ix->hctl_d;
   c.ctl = ix->ctl;
-  c.arr = Queue{(u32 *)ix->arr_buf, ix->ring_cap - 1, &ix->ctl->q_heads[0], &ix->ctl->q_heads[1]};
-  c.run = Queue{(u32 *)ix->run_buf, ix->runq_cap - 1, &ix->ctl->q_heads[2], &ix->ctl->q_heads[3]};
-  c.retry = Queue{(u32 *)ix->retry_buf, ix->runq_cap - 1, &ix->ctl->q_heads[4], &ix->ctl->q_heads[5]};
+  u32 *qh = ix->ctl->q_heads;
+  c.arr = Queue{(u32 *)ix->arr_buf, ix->arr_cap - 1, qh + 0, qh + 1, (int *)(qh + 2)};
+  c.run = Queue{(u32 *)ix->run_buf, ix->runq_cap - 1, qh + 3, qh + 4, (int *)(qh + 5)};
+  c.want = Queue{(u32 *)ix->want_buf, ix->want_cap - 1, qh + 6, qh + 7, (int *)(qh + 8)};
   c.nq = nq; c.K = K; c.L = L; c.W = W; c.WR = ix->qs_WR;
   c.queries = queries_dev; c.out_ids = out_ids_dev; c.out_dists = out_dists_dev;
   c.out_pages = out_pages_distinct_dev; c.out_counters = out_counters_dev;
@@ -535,10 +541,10 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
     const u32 s = h.status ? h.status : (u32)GORIO_ERR_INTERNAL;
     std::snprintf(buf, sizeof buf,
                   "device: %s (site 0x%x, %u, %u, %u; block %u thread %u; done %u/%u; posted %u; arrivals %u/%u; "
-                  "runnable %u/%u; retry %u/%u; proxy consumed %u published %u outstanding %u queued %u "
+                  "runnable %u/%u; want %u/%u; proxy consumed %u published %u outstanding %u queued %u "
                   "[head stream %u seq %u copied %u])",
                   s < 9 ? kDeviceErr[s] : "?", h.dbg[0], h.dbg[1], h.dbg[2], h.dbg[3], h.dbg[4], h.dbg[5], h.done, nq,
-                  h.ring_head, h.q_heads[0], h.q_heads[1], h.q_heads[2], h.q_heads[3], h.q_heads[4], h.q_heads[5],
+                  h.ring_head, h.q_heads[0], h.q_heads[1], h.q_heads[3], h.q_heads[4], h.q_heads[6], h.q_heads[7],
                   ix->px_dbg[0], ix->px_dbg[1], ix->px_dbg[2], ix->px_dbg[3], ix->px_dbg[4], ix->px_dbg[5], ix->px_dbg[6]);
     return fail(ix, (int)s, buf);
   }

@@ -12,16 +12,12 @@ typedef uint32_t u32;
 typedef uint64_t u64;
 
 constexpr u32 kPageBytes = 4096;
-constexpr u32 kWays = 16;             // set associativity of the page cache
 constexpr u32 kNil = 0xFFFFFFFFu;     // end of a waiter list
 constexpr u32 kClosed = 0xFFFFFFFEu;  // waiter list closed: the page has arrived
 constexpr u32 kInvalidId = 0xFFFFFFFFu;
 constexpr u64 kPadKey = ~0ull;        // sorts after every real key
 constexpr u32 kMaxFillBatch = 128;
 constexpr u32 kPqKsub = 256;
-
-// Slot tag word: [page:32][generation:28][ref:1][state:3]
-enum SlotState : u32 { ST_EMPTY = 0, ST_RESERVED = 1, ST_FILLING = 2, ST_ARRIVED = 3, ST_READY = 4 };
 
 // Query phases: which batch of page items is outstanding for the query slot.
 enum Phase : u32 { PH_NEW = 0, PH_EVAL = 1, PH_EXPAND = 2 };
@@ -33,19 +29,26 @@ struct QHdr {
   u32 phase;
   u32 awaiting;   // outstanding items of the current batch (+1 guard while issuing/retrying)
   u32 n_items;    // items in the current batch
-  u32 n_todo;     // items of the batch whose lookup must be retried
+  u32 reserved0;
   u32 list_len;
   u32 n_iter, n_expand, n_eval, sum_deg, pages_distinct;
   u32 pool_len;   // PQ mode: entries in the rerank pool
   u32 pad[4];
 };
 
-// Multi-producer multi-consumer ring of u32 values in HBM (cells hold value+1, 0 = empty).
+// Multi-producer multi-consumer ring of u32 values in HBM (cells hold sequence << 32 | value).
 struct Queue {
   u32 *buf;
   u32 mask;
   u32 *head;
   u32 *tail;
+  int *count;   // items pushed minus items claimed by consumers
+};
+
+// Clock hand and never-used-slot bump pointer of the page cache.
+struct CacheShared {
+  u32 hand;
+  u32 bump;
 };
 
 // Device-resident control block.
@@ -55,7 +58,7 @@ struct Ctl {
   u32 next_query;  // next query id to admit when a slot frees
   u32 done;        // queries finished
   u32 ring_head;   // request descriptors posted
-  u32 q_heads[8];  // queue head/tail words: arr(0,1) run(2,3) retry(4,5)
+  u32 q_heads[12]; // queue head/tail/count words: arr(0,1,2) run(3,4,5) want(6,7,8)
   u32 dbg[8];      // detail of the first error
   u64 stats[16];
 };
@@ -71,11 +74,12 @@ struct Ctx {
   const u8 *pq_cent;
   const u8 *pq_codes;
   // page cache
-  u8 *slot_data;   // n_slots * 4096, slot = way * n_sets + set
-  u64 *tag;        // [n_sets][kWays]
-  u64 *wl;         // [n_sets][kWays]  (generation << 32 | waiter list head)
-  u32 *hand;       // [n_sets] clock hands
-  u32 n_sets, n_slots;
+  u8 *slot_data;   // n_slots * 4096
+  u64 *ptab;       // [n_pages] page words: state, slot, waiter-list head or generation
+  u64 *smeta;      // [n_slots] slot words: page, generation, reference bit
+  u32 *parts;      // [n_slots] waiter-chain segments still being served
+  CacheShared *cs; // clock hand and bump pointer
+  u32 n_slots;
   // miss ring: host-mapped, written by the GPU, consumed by the proxy
   u64 *ring;
   u32 ring_mask, ring_shift;
@@ -83,7 +87,7 @@ struct Ctx {
   const u32 *comp_ring;
   u32 comp_mask;
   const u32 *host_ctl;  // [0] completion tail, [1] abort request
-  Queue arr, run, retry;
+  Queue arr, run, want;   // arrivals (slots / chain continuations), runnable query slots, pages awaiting a slot
   // query state
   u32 n_qslots, nq, K, L, W, WR;
   QHdr *hdr;
@@ -93,7 +97,6 @@ struct Ctx {
   u32 *wrec;     // [n_qslots][WR] next pointers of waiter records (record id = qs*WR + j)
   u32 *adj;      // [n_qslots][W][R]
   u32 *adjdeg;   // [n_qslots][W]
-  u16 *todo;     // [n_qslots][WR]
   u32 *seen;     // [n_qslots][seen_cap]
   u32 *pset;     // [n_qslots][pset_cap]
   u64 *pool;     // [n_qslots][K + W]   PQ rerank pool (sorted, <= K kept)

@@ -79,36 +79,40 @@ __device__ __forceinline__ void stat_add(const Ctx &c, u32 idx, u32 v) {
 // ------------------------------------------------------------------------------------------
 // bounded MPMC queue of u32 (cells = sequence << 32 | value); one lane calls these
 // ------------------------------------------------------------------------------------------
+// Tickets are taken with fetch-and-add on both ends, never with compare-and-swap loops:
+// thousands of warps poll these queues, and a CAS on a shared head lets only one of them
+// through per L2 round trip.  A signed item count guards the consumer side: a consumer
+// first takes one unit of the count (backing out if there was none), and only then a head
+// ticket, so a ticket is always for a cell whose producer has at least reserved it; the wait
+// for that cell is bounded by the producer's own push.
 constexpr u32 kSpinLimit = 1u << 22;
 
 __device__ void q_push(const Ctx &c, const Queue &q, u32 v) {
   __threadfence();   // everything written for the consumer is visible before the cell
-  u32 pos = atomicAdd(q.tail, 1u);
+  const u32 pos = atomicAdd(q.tail, 1u);
   u64 *cell = (u64 *)q.buf + (pos & q.mask);
   u32 spins = 0;
   while ((u32)(ld_u64(cell) >> 32) != pos) {      // previous lap's consumer not done yet
     if (++spins > kSpinLimit) { raise(c, 8, 0x51, pos); return; }
   }
   st_u64(cell, ((u64)(pos + 1u) << 32) | v);
+  atomicAdd(q.count, 1);
 }
 
 __device__ bool q_pop(const Ctx &c, const Queue &q, u32 &out) {
-  for (int tries = 0; tries < 8; ++tries) {
-    u32 h = ld_u32(q.head), t = ld_u32(q.tail);
-    if ((int)(t - h) <= 0) return false;
-    if (atomicCAS(q.head, h, h + 1u) != h) continue;
-    u64 *cell = (u64 *)q.buf + (h & q.mask);
-    u32 spins = 0;
-    u64 v;
-    while ((u32)((v = ld_u64(cell)) >> 32) != h + 1u) {
-      if (++spins > kSpinLimit) { raise(c, 8, 0x52, h); return false; }
-    }
-    st_u64(cell, (u64)(h + q.mask + 1u) << 32);
-    __threadfence();
-    out = (u32)v;
-    return true;
+  if ((int)ld_u32((const u32 *)q.count) <= 0) return false;
+  if (atomicSub(q.count, 1) <= 0) { atomicAdd(q.count, 1); return false; }
+  const u32 h = atomicAdd(q.head, 1u);
+  u64 *cell = (u64 *)q.buf + (h & q.mask);
+  u32 spins = 0;
+  u64 v;
+  while ((u32)((v = ld_u64(cell)) >> 32) != h + 1u) {
+    if (++spins > kSpinLimit) { raise(c, 8, 0x52, h); return false; }
   }
-  return false;
+  st_u64(cell, (u64)(h + q.mask + 1u) << 32);
+  __threadfence();
+  out = (u32)v;
+  return true;
 }
 
 // warp-level pop: lane 0 pops, the result is broadcast
@@ -121,21 +125,29 @@ __device__ __forceinline__ bool warp_pop(const Ctx &c, const Queue &q, u32 &out,
 }
 
 // ------------------------------------------------------------------------------------------
-// slot tags
+// page cache and miss tracker
 // ------------------------------------------------------------------------------------------
-constexpr u64 kRefBit = 8ull;
-__device__ __forceinline__ u64 mk_tag(u32 page, u32 gen, u32 ref, u32 state) {
-  return ((u64)page << 32) | ((u64)(gen & 0x0FFFFFFFu) << 4) | ((u64)ref << 3) | state;
+// One 64-bit word per index page is the single point of truth for that page:
+//   [state:3][slot:29][low:32]   low = head of the page's waiter list (WANTED, FILLING)
+//                                      or the slot's fill generation (ARRIVED, RESIDENT)
+//   ABSENT   nobody wants the page               WANTED  waiters, no slot yet (queued in want_q)
+//   FILLING  slot assigned, request posted       ARRIVED data present, waiters being served
+//   RESIDENT data present, evictable
+// It is a hash of page -> slot with the identity hash (page ids are dense and known at open),
+// so a lookup is one load and the first miss on a page is decided by one compare-and-swap:
+// concurrent misses on the same page, from any lane of any query, can only join its list.
+// One 64-bit word per slot ([page:32][generation:31][ref:1]) serves the clock.
+enum PageState : u32 { P_ABSENT = 0, P_WANTED = 1, P_FILLING = 2, P_ARRIVED = 3, P_RESIDENT = 4 };
+constexpr u64 kAbsentWord = (u64)kNil;
+__device__ __forceinline__ u64 mk_pw(u32 state, u32 slot, u32 low) {
+  return ((u64)state << 61) | ((u64)slot << 32) | low;
 }
-__device__ __forceinline__ u32 tag_page(u64 t) { return (u32)(t >> 32); }
-__device__ __forceinline__ u32 tag_gen(u64 t) { return (u32)(t >> 4) & 0x0FFFFFFFu; }
-__device__ __forceinline__ u32 tag_state(u64 t) { return (u32)t & 7u; }
-__device__ __forceinline__ u32 slot_of(const Ctx &c, u32 ti) { return (ti % kWays) * c.n_sets + ti / kWays; }
-__device__ __forceinline__ u32 ti_of(const Ctx &c, u32 slot) { return (slot % c.n_sets) * kWays + slot / c.n_sets; }
-
-// lookup result: [gen:28 | pad][ti:29][code:3]
-enum LookupCode : u32 { LK_NONE = 0, LK_HIT = 1, LK_WAIT = 2, LK_DEFER = 3 };
-__device__ __forceinline__ u64 mk_res(u32 code, u32 ti, u32 gen) { return ((u64)gen << 32) | ((u64)ti << 3) | code; }
+__device__ __forceinline__ u32 pw_state(u64 w) { return (u32)(w >> 61); }
+__device__ __forceinline__ u32 pw_slot(u64 w) { return (u32)(w >> 32) & 0x1FFFFFFFu; }
+__device__ __forceinline__ u32 pw_low(u64 w) { return (u32)w; }
+__device__ __forceinline__ u64 mk_sm(u32 page, u32 gen, u32 ref) { return ((u64)page << 32) | ((u64)(gen & 0x7FFFFFFFu) << 1) | ref; }
+__device__ __forceinline__ u32 sm_page(u64 m) { return (u32)(m >> 32); }
+__device__ __forceinline__ u32 sm_gen(u64 m) { return (u32)(m >> 1) & 0x7FFFFFFFu; }
 
 struct LaneStats { u32 hit, missed, joins, evict, retry, posted; };
 
@@ -150,96 +162,84 @@ __device__ __forceinline__ void post_request(const Ctx &c, u32 page, u32 slot) {
   st_sys_u64(c.ring + (idx & c.ring_mask), ((u64)page << 32) | ((u64)slot << 8) | lap);
 }
 
-// Page lookup / miss generation by ONE lane (lanes of a warp that want the same page elect a
-// leader first, so a warp never races with itself).
-__device__ u64 cache_lookup(const Ctx &c, u32 page, LaneStats &st) {
-  const u32 set = page % c.n_sets;
-  u64 *tags = c.tag + (u64)set * kWays;
-  for (int attempt = 0; attempt < 24; ++attempt) {
-    // 1. scan the set
-    int found = -1; u64 ft = 0;
-#pragma unroll
-    for (int w = 0; w < (int)kWays; ++w) {
-      u64 t = ld_u64(tags + w);
-      if (tag_page(t) == page && tag_state(t) != ST_EMPTY && found < 0) { found = w; ft = t; }
-    }
-    if (found >= 0) {
-      u32 s = tag_state(ft), ti = set * kWays + found;
-      if (s == ST_READY || s == ST_ARRIVED) return mk_res(LK_HIT, ti, tag_gen(ft));
-      if (s == ST_FILLING) return mk_res(LK_WAIT, ti, tag_gen(ft));
-      __nanosleep(64);           // RESERVED: another lane is deciding a race on this page
-      continue;
-    }
-    // 2. miss: claim a victim with the set's clock hand
-    // The page's home way ((page / n_sets) % ways) is tried first while it is empty: rival
-    // claims for one page then meet on a single compare-and-swap, and with capacity for
-    // every page each page has a way of its own, so nothing is ever evicted or fetched twice.
-    int victim = -1; u32 vgen = 0;
-    {
-      const u32 w = (page / c.n_sets) % kWays;
-      const u64 t = ld_u64(tags + w);
-      if (tag_state(t) == ST_EMPTY) {
-        const u64 nt = mk_tag(page, tag_gen(t) + 1u, 0, ST_RESERVED);
-        if (atomicCAS((unsigned long long *)(tags + w), t, nt) != t) continue;   // lost the race: rescan
-        victim = (int)w; vgen = tag_gen(nt);
-      } else if (tag_page(t) == page) {
-        continue;                                   // the page appeared meanwhile: rescan
-      }
-    }
-    // otherwise the set's clock hand picks a victim: second chance for referenced pages
-    for (int step = 0; victim < 0 && step < 3 * (int)kWays; ++step) {
-      const u32 w = atomicAdd(c.hand + set, 1u) % kWays;
-      const u64 t = ld_u64(tags + w);
-      const u32 s = tag_state(t);
-      if (s == ST_EMPTY || (s == ST_READY && !(t & kRefBit))) {
-        const u64 nt = mk_tag(page, tag_gen(t) + 1u, 0, ST_RESERVED);
-        if (atomicCAS((unsigned long long *)(tags + w), t, nt) == t) {
-          victim = (int)w; vgen = tag_gen(nt);
-          if (s == ST_READY) st.evict++;
-        }
-      } else if (s == ST_READY) {
-        atomicCAS((unsigned long long *)(tags + w), t, t & ~kRefBit);
-      }
-    }
-    if (victim < 0) return mk_res(LK_DEFER, 0, 0);     // every way is in flight: retry later
-    // 3. another lane may have claimed a way for the same page concurrently: whoever sees
-    //    a rival backs off, so at most one claim per page survives
-    fence_sc();
-    bool rival = false;
-#pragma unroll
-    for (int w = 0; w < (int)kWays; ++w) {
-      u64 t = ld_u64(tags + w);
-      if (w != victim && tag_page(t) == page && tag_state(t) != ST_EMPTY) rival = true;
-    }
-    const u32 ti = set * kWays + (u32)victim;
-    if (rival) {
-      st_u64(tags + victim, mk_tag(kInvalidId, vgen, 0, ST_EMPTY));
-      __nanosleep(32 + 16 * (lane_id() & 7u));
-      continue;
-    }
-    // 4. won: open the waiter list, publish FILLING, post the descriptor
-    st_u64(c.wl + ti, ((u64)vgen << 32) | kNil);
-    __threadfence();
-    st_u64(tags + victim, mk_tag(page, vgen, 0, ST_FILLING));
-    __threadfence_system();      // the tag must be visible to whoever learns of the request
-    post_request(c, page, slot_of(c, ti));
-    st.posted++;
-    return mk_res(LK_WAIT, ti, vgen) | (1ull << 63);    // bit 63: this lane is the owner
+// Get a slot for a new page: never-used slots first, then the clock (second chance for
+// referenced pages); `hint` (a slot the caller has just made evictable) is taken if a short
+// sweep finds nothing.  Returns kNil when every slot examined is in flight.
+__device__ u32 alloc_slot(const Ctx &c, u32 hint, LaneStats &st) {
+  if (ld_u32(&c.cs->bump) < c.n_slots) {
+    u32 b = atomicAdd(&c.cs->bump, 1u);
+    if (b < c.n_slots) return b;
   }
-  return mk_res(LK_DEFER, 0, 0);
+  const int sweep = hint != kNil ? 8 : 48;
+  for (int step = 0; step <= sweep; ++step) {
+    const bool use_hint = step == sweep;
+    if (use_hint && hint == kNil) break;
+    const u32 s = use_hint ? hint : atomicAdd(&c.cs->hand, 1u) % c.n_slots;
+    const u64 m = ld_u64(c.smeta + s);
+    const u32 pg = sm_page(m);
+    if (pg >= c.n_pages) continue;                       // slot handed out but not yet labelled
+    const u64 w = ld_u64(c.ptab + pg);
+    if (pw_state(w) != P_RESIDENT || pw_slot(w) != s) continue;
+    if ((m & 1ull) && !use_hint) {                       // referenced: second chance
+      atomicCAS((unsigned long long *)(c.smeta + s), m, m & ~1ull);
+      continue;
+    }
+    if (atomicCAS((unsigned long long *)(c.ptab + pg), w, kAbsentWord) == w) { st.evict++; return s; }
+  }
+  return kNil;
 }
 
-// Link waiter record g (= query slot * WR + item) into the slot's list.
-__device__ bool register_waiter(const Ctx &c, u32 ti, u32 gen, u32 g) {
-  u64 *wl = c.wl + ti;
-  for (int tries = 0; tries < 128; ++tries) {
-    u64 cur = ld_u64(wl);
-    if ((u32)(cur >> 32) != gen || (u32)cur == kClosed) return false;
-    st_u32(c.wrec + g, (u32)cur);
-    __threadfence();
-    if (atomicCAS((unsigned long long *)wl, cur, ((u64)gen << 32) | g) == cur) return true;
+// The page is WANTED and `slot` is exclusively ours: label the slot, move the page to
+// FILLING (keeping whatever waiters have queued up meanwhile) and post the descriptor.
+__device__ void assign_and_post(const Ctx &c, u32 page, u32 slot, LaneStats &st) {
+  const u32 gen = sm_gen(ld_u64(c.smeta + slot)) + 1u;
+  st_u64(c.smeta + slot, mk_sm(page, gen, 0));
+  __threadfence();
+  for (u32 spins = 0;; ++spins) {
+    const u64 w = ld_u64(c.ptab + page);
+    if (pw_state(w) != P_WANTED || spins > kSpinLimit) { raise(c, 8, 0x41, page, (u32)(w >> 32), spins); return; }
+    if (atomicCAS((unsigned long long *)(c.ptab + page), w, mk_pw(P_FILLING, slot, pw_low(w))) == w) break;
   }
-  return false;
+  __threadfence_system();      // page word and slot label visible to whoever learns of the request
+  post_request(c, page, slot);
+  st.posted++;
+}
+
+// Serve one page from the want queue if a slot can be had (one lane).
+__device__ void serve_want(const Ctx &c, u32 hint, LaneStats &st) {
+  u32 page;
+  if (!q_pop(c, c.want, page)) return;
+  const u32 slot = alloc_slot(c, hint, st);
+  if (slot == kNil) { q_push(c, c.want, page); return; }
+  assign_and_post(c, page, slot, st);
+}
+
+// Lookup / miss generation for one item by one lane.  g is the item's waiter record.
+// Returns LK_HIT with (slot, generation) to be consumed and validated by the caller, or
+// LK_WAIT when the item now waits on the page (as first requester or as a joiner).
+enum LookupCode : u32 { LK_NONE = 0, LK_HIT = 1, LK_WAIT = 2 };
+__device__ u32 page_lookup(const Ctx &c, u32 page, u32 g, u32 &slot, u32 &gen, LaneStats &st) {
+  u64 *pw = c.ptab + page;
+  for (u32 tries = 0; tries < 4096; ++tries) {
+    const u64 w = ld_u64(pw);
+    const u32 s = pw_state(w);
+    if (s == P_RESIDENT || s == P_ARRIVED) { slot = pw_slot(w); gen = pw_low(w); return LK_HIT; }
+    st_u32(c.wrec + g, s == P_ABSENT ? kNil : pw_low(w));
+    __threadfence();
+    if (s == P_ABSENT) {
+      if (atomicCAS((unsigned long long *)pw, w, mk_pw(P_WANTED, 0, g)) != w) continue;
+      st.missed++;
+      const u32 sl = alloc_slot(c, kNil, st);          // first requester: find the page a slot
+      if (sl != kNil) assign_and_post(c, page, sl, st);
+      else q_push(c, c.want, page);
+      return LK_WAIT;
+    }
+    if (atomicCAS((unsigned long long *)pw, w, (w & 0xFFFFFFFF00000000ull) | g) != w) continue;
+    st.missed++; st.joins++;
+    return LK_WAIT;
+  }
+  raise(c, 8, 0x42, page, g);
+  return LK_WAIT;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -307,38 +307,87 @@ __device__ __forceinline__ void complete_items(const Ctx &c, u32 qs, u32 n) {
   else if (old < n) raise(c, 8, 0x61, qs, old, n);
 }
 
-// A page has arrived in `slot`: consume it for every registered waiter, then make it
-// evictable.  (Section 3.2: the per-slot ready entry is what the GPU tests on resume.)
-__device__ void consume_arrival(const Ctx &c, u32 slot, u32 lane) {
-  if (slot >= c.n_slots) { if (lane == 0) raise(c, 8, 0x71, slot); return; }
-  const u32 ti = ti_of(c, slot);
-  u64 t = ld_u64(c.tag + ti);
-  t = __shfl_sync(0xffffffffu, t, 0);
-  if (tag_state(t) != ST_FILLING) { if (lane == 0) raise(c, 8, 0x72, slot, (u32)t, (u32)(t >> 32)); return; }
-  const u32 page = tag_page(t), gen = tag_gen(t);
-  u32 head = 0;
+// Waiter lists can be long (every query waits on the entry page at the start), so a warp
+// consumes at most kChainSegment records and hands the rest of the chain to another warp
+// through the arrival queue; `parts` counts the segments still being served for the slot.
+constexpr u32 kChainSegment = 32;
+constexpr u32 kContFlag = 0x80000000u;
+
+__device__ void finish_arrival(const Ctx &c, u32 slot, u32 page, u32 gen, u32 lane) {
+  // last segment done: the page becomes evictable, and the slot's turn-over feeds the
+  // pages that are waiting for a slot
   if (lane == 0) {
-    st_u64(c.tag + ti, mk_tag(page, gen, 1, ST_ARRIVED));
     __threadfence();
-    u64 old = atomicExch((unsigned long long *)(c.wl + ti), ((u64)gen << 32) | kClosed);
-    head = (u32)old;
-    __threadfence();
+    st_u64(c.ptab + page, mk_pw(P_RESIDENT, slot, gen));
+    LaneStats st = {0, 0, 0, 0, 0, 0};
+    serve_want(c, slot, st);
+    stat_add(c, S_EVICT, st.evict); stat_add(c, S_POSTED, st.posted);
   }
-  head = __shfl_sync(0xffffffffu, head, 0);
-  u32 g = head, count = 0;
+  __syncwarp();
+}
+
+// Consume the waiter chain starting at record g for the page held in `slot`.
+__device__ void consume_chain(const Ctx &c, u32 slot, u32 page, u32 gen, u32 g, u32 lane) {
   const u32 limit = c.n_qslots * c.WR;
-  while (g != kNil) {
-    if (g >= limit || ++count > limit) { if (lane == 0) raise(c, 8, 0x73, slot, g, count); return; }
-    const u32 next = ld_u32(c.wrec + g);
-    const u32 qs = g / c.WR, j = g % c.WR;
+  // chase up to a segment of next pointers first so that the remainder is handed off early
+  u32 mine = kNil, n = 0, cur = g;
+  while (cur != kNil && n < kChainSegment) {
+    if (cur >= limit) { if (lane == 0) raise(c, 8, 0x73, slot, cur, n); return; }
+    if (lane == n) mine = cur;
+    cur = uld(c.wrec + cur);
+    ++n;
+  }
+  if (cur != kNil && lane == 0) {
+    atomicAdd(c.parts + slot, 1u);
+    q_push(c, c.arr, kContFlag | cur);
+  }
+  for (u32 i = 0; i < n; ++i) {
+    const u32 rec = __shfl_sync(0xffffffffu, mine, i);
+    const u32 qs = rec / c.WR, j = rec % c.WR;
     consume_item(c, qs, j, slot, lane);
     __threadfence();      // every lane's result stores before lane 0 counts the item done
     __syncwarp();
     if (lane == 0) complete_items(c, qs, 1);
-    g = next;
   }
-  __syncwarp();
-  if (lane == 0) { __threadfence(); st_u64(c.tag + ti, mk_tag(page, gen, 1, ST_READY)); }
+  u32 last = 0;
+  if (lane == 0) last = atomicSub(c.parts + slot, 1u) == 1u ? 1u : 0u;
+  if (__shfl_sync(0xffffffffu, last, 0)) finish_arrival(c, slot, page, gen, lane);
+}
+
+// A page has arrived in `slot` (Section 3.2: the per-slot ready entry): take its waiter
+// list, serve it, then make the page evictable.  v is a slot id, or a continuation
+// (kContFlag | record) of a chain another warp handed off.
+__device__ void consume_arrival(const Ctx &c, u32 v, u32 lane) {
+  if (v & kContFlag) {
+    const u32 g = v & ~kContFlag;
+    if (g >= c.n_qslots * c.WR) { if (lane == 0) raise(c, 8, 0x74, g); return; }
+    const u32 node = uld(c.items + g);
+    const u32 page = node / c.npp;
+    u64 w = ld_u64(c.ptab + page);
+    w = __shfl_sync(0xffffffffu, w, 0);
+    if (pw_state(w) != P_ARRIVED) { if (lane == 0) raise(c, 8, 0x75, g, page, (u32)(w >> 32)); return; }
+    consume_chain(c, pw_slot(w), page, pw_low(w), g, lane);
+    return;
+  }
+  const u32 slot = v;
+  if (slot >= c.n_slots) { if (lane == 0) raise(c, 8, 0x71, slot); return; }
+  u64 m = ld_u64(c.smeta + slot);
+  m = __shfl_sync(0xffffffffu, m, 0);
+  const u32 page = sm_page(m), gen = sm_gen(m);
+  if (page >= c.n_pages) { if (lane == 0) raise(c, 8, 0x76, slot, page); return; }
+  u32 head = 0, bad = 0;
+  if (lane == 0) {
+    st_u32(c.parts + slot, 1u);
+    st_u64(c.smeta + slot, m | 1ull);                      // a fresh page gets its second chance
+    __threadfence();
+    const u64 old = atomicExch((unsigned long long *)(c.ptab + page), mk_pw(P_ARRIVED, slot, gen));
+    if (pw_state(old) != P_FILLING || pw_slot(old) != slot) { raise(c, 8, 0x72, slot, page, (u32)(old >> 32)); bad = 1; }
+    head = pw_low(old);
+    __threadfence();
+  }
+  if (__shfl_sync(0xffffffffu, bad, 0)) return;
+  head = __shfl_sync(0xffffffffu, head, 0);
+  consume_chain(c, slot, page, gen, head, lane);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -361,32 +410,29 @@ __device__ u32 set_insert(u32 *tab, u32 cap, u32 v) {
 // ------------------------------------------------------------------------------------------
 // issue a batch of page items for query slot qs
 // ------------------------------------------------------------------------------------------
-// from_todo = false: items 0..n_items-1 of the current batch, `awaiting` is armed here.
-// from_todo = true : retry the deferred items listed in todo[0..n_todo).
-// Returns true if the whole batch is complete (the caller goes on inline); false if the
-// query was parked (someone else resumes it) or re-queued for a retry.
-__device__ bool issue_batch(const Ctx &c, u32 qs, bool from_todo, u32 lane) {
+// Items 0..n_items-1 of the current batch: every lane looks its item's page up; hits are
+// consumed now (warp cooperative) and validated against the page word afterwards; misses
+// leave the item waiting on the page.  Returns true if the whole batch completed inline
+// (the caller goes on with the next phase), false if the query is parked: whoever
+// consumes its last item pushes it back onto the runnable queue.
+__device__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
   QHdr *h = c.hdr + qs;
   const u32 phase = uld(&h->phase);
-  const u32 n = from_todo ? uld(&h->n_todo) : uld(&h->n_items);
-  const bool count_pages = !from_todo && ((c.pq_m == 0) == (phase == PH_EVAL));
-  if (!from_todo) {
-    if (lane == 0) st_u32(&h->awaiting, n + 1u);
-  }
+  const u32 n = uld(&h->n_items);
+  const bool count_pages = (c.pq_m == 0) == (phase == PH_EVAL);
+  if (lane == 0) st_u32(&h->awaiting, n + 1u);      // +1: guard held until everything is issued
   __threadfence();
   __syncwarp();
-  u16 *todo = c.todo + (u64)qs * c.WR;
   const u32 *items = c.items + (u64)qs * c.WR;
   u32 *pset = c.pset + (u64)qs * c.pset_cap;
   LaneStats st = {0, 0, 0, 0, 0, 0};
-  u32 n_done = 0, n_todo_new = 0, new_pages = 0;
+  u32 n_done = 0, new_pages = 0;
 
   for (u32 base = 0; base < n; base += 32) {
-    const u32 idx = base + lane;
-    const bool active = idx < n;
-    u32 j = 0, node = 0, page = kInvalidId;
-    if (active) {
-      j = from_todo ? (u32)ld_u16(todo + idx) : idx;
+    const u32 j = base + lane;
+    bool pending = j < n;
+    u32 node = 0, page = kInvalidId;
+    if (pending) {
       node = ld_u32(items + j);
       page = node / c.npp;
       if (count_pages) {
@@ -395,59 +441,38 @@ __device__ bool issue_batch(const Ctx &c, u32 qs, bool from_todo, u32 lane) {
         else if (r == 2) raise(c, 6, 0x81, qs, page);
       }
     }
-    __syncwarp();
-    // lanes that want the same page elect the lowest lane as leader
-    const u32 amask = __ballot_sync(0xffffffffu, active);
-    u64 res = 0;
-    u32 leader = lane;
-    if (active) {
-      u32 grp = __match_any_sync(amask, page);
-      leader = __ffs(grp) - 1;
-      if (leader == lane) res = cache_lookup(c, page, st);
-    }
-    __syncwarp();
-    res = __shfl_sync(0xffffffffu, res, leader);
-    u32 code = active ? (u32)(res & 7u) : LK_NONE;
-    const u32 ti = (u32)((res & 0xFFFFFFFFull) >> 3), gen = (u32)(res >> 32) & 0x0FFFFFFFu;
-    const bool owner = (res >> 63) && leader == lane;
-    if (code == LK_WAIT) {
-      if (register_waiter(c, ti, gen, qs * c.WR + j)) { st.missed++; if (!owner) st.joins++; }
-      else code = LK_DEFER;
-    }
-    // hits: consume now (warp cooperative, one item at a time), then validate the tags
-    u32 hits = __ballot_sync(0xffffffffu, code == LK_HIT);
-    for (u32 m = hits; m; m &= m - 1) {
-      const u32 src = __ffs(m) - 1;
-      const u32 sj = __shfl_sync(0xffffffffu, j, src);
-      const u32 sti = __shfl_sync(0xffffffffu, ti, src);
-      consume_item(c, qs, sj, slot_of(c, sti), lane);
-    }
-    if (hits) {
-      __threadfence();
-      if (code == LK_HIT) {
-        u64 t2 = ld_u64(c.tag + ti);
-        const u32 s2 = tag_state(t2);
-        if (tag_page(t2) == page && tag_gen(t2) == gen && (s2 == ST_READY || s2 == ST_ARRIVED)) {
-          if (!(t2 & kRefBit)) atomicCAS((unsigned long long *)(c.tag + ti), t2, t2 | kRefBit);
-          st.hit++; n_done++;
-        } else {
-          code = LK_DEFER;     // evicted while we were reading: the item is redone later
+    for (u32 round = 0; __any_sync(0xffffffffu, pending); ++round) {
+      u32 code = LK_NONE, slot = 0, gen = 0;
+      if (pending) code = page_lookup(c, page, qs * c.WR + j, slot, gen, st);
+      __syncwarp();
+      if (code == LK_WAIT) pending = false;
+      const u32 hits = __ballot_sync(0xffffffffu, code == LK_HIT);
+      for (u32 m = hits; m; m &= m - 1) {
+        const u32 src = __ffs(m) - 1;
+        consume_item(c, qs, __shfl_sync(0xffffffffu, j, src), __shfl_sync(0xffffffffu, slot, src), lane);
+      }
+      if (hits) {
+        __threadfence();
+        if (code == LK_HIT) {
+          // the bytes just read were the page's if its word still names this slot and fill
+          const u64 w2 = ld_u64(c.ptab + page);
+          const u32 s2 = pw_state(w2);
+          if ((s2 == P_RESIDENT || s2 == P_ARRIVED) && pw_slot(w2) == slot && pw_low(w2) == gen) {
+            const u64 m2 = ld_u64(c.smeta + slot);
+            if (!(m2 & 1ull)) atomicCAS((unsigned long long *)(c.smeta + slot), m2, m2 | 1ull);
+            st.hit++; n_done++;
+            pending = false;
+          } else {
+            st.retry++;              // evicted under the read: look the page up again
+          }
         }
       }
+      if (round > 1024) { if (lane == 0) raise(c, 8, 0x84, qs, base); break; }
+      if (warp_stopped(c)) break;
     }
-    // deferred items go (back) on the todo list; in-place compaction is safe because every
-    // lane has already read its entry of this round
-    __syncwarp();
-    const u32 defer = __ballot_sync(0xffffffffu, code == LK_DEFER);
-    if (code == LK_DEFER) {
-      st_u16(todo + n_todo_new + __popc(defer & ((1u << lane) - 1u)), (u16)j);
-      st.retry++;
-    }
-    n_todo_new += __popc(defer);
     if (warp_stopped(c)) break;
   }
 
-  // warp totals
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     n_done += __shfl_xor_sync(0xffffffffu, n_done, o);
@@ -466,21 +491,10 @@ __device__ bool issue_batch(const Ctx &c, u32 qs, bool from_todo, u32 lane) {
     stat_add(c, S_HIT, st.hit); stat_add(c, S_MISSED, st.missed); stat_add(c, S_JOINS, st.joins);
     stat_add(c, S_EVICT, st.evict); stat_add(c, S_RETRY, st.retry); stat_add(c, S_POSTED, st.posted);
     if (new_pages) st_u32(&h->pages_distinct, ld_u32(&h->pages_distinct) + new_pages);
-    if (n_todo_new == 0) {
-      st_u32(&h->n_todo, 0);
-      __threadfence();
-      u32 old = atomicSub(&h->awaiting, n_done + 1u);       // drop the guard too
-      if (old == n_done + 1u) complete = 1;
-      else if (old < n_done + 1u) raise(c, 8, 0x82, qs, old, n_done);
-    } else {
-      st_u32(&h->n_todo, n_todo_new);
-      __threadfence();
-      if (n_done) {
-        u32 old = atomicSub(&h->awaiting, n_done);           // the guard stays
-        if (old <= n_done) raise(c, 8, 0x83, qs, old, n_done);
-      }
-      q_push(c, c.retry, qs);
-    }
+    __threadfence();
+    const u32 old = atomicSub(&h->awaiting, n_done + 1u);       // inline hits and the guard
+    if (old == n_done + 1u) complete = 1;
+    else if (old < n_done + 1u) raise(c, 8, 0x82, qs, old, n_done);
   }
   return __shfl_sync(0xffffffffu, complete, 0) != 0u;
 }
@@ -737,7 +751,7 @@ __device__ void finish_query(const Ctx &c, u32 qs, u32 lane) {
 
 __device__ __forceinline__ void reset_hdr(QHdr *h, u32 qid) {
   st_u32(&h->qid, qid); st_u32(&h->phase, PH_NEW); st_u32(&h->awaiting, 0); st_u32(&h->n_items, 0);
-  st_u32(&h->n_todo, 0); st_u32(&h->list_len, 0); st_u32(&h->n_iter, 0); st_u32(&h->n_expand, 0);
+  st_u32(&h->reserved0, 0); st_u32(&h->list_len, 0); st_u32(&h->n_iter, 0); st_u32(&h->n_expand, 0);
   st_u32(&h->n_eval, 0); st_u32(&h->sum_deg, 0); st_u32(&h->pages_distinct, 0); st_u32(&h->pool_len, 0);
 }
 
@@ -759,11 +773,8 @@ __device__ bool recycle_slot(const Ctx &c, u32 qs, u32 lane) {
 }
 
 template <bool PQ>
-__device__ void run_query(const Ctx &c, u32 qs, bool retry, u32 lane, u32 *lut) {
+__device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut) {
   QHdr *h = c.hdr + qs;
-  if (retry) {
-    if (!issue_batch(c, qs, true, lane)) return;
-  }
   for (u32 guard = 0; guard < 4u * c.max_iters + 64u; ++guard) {
     if (warp_stopped(c)) return;
     const u32 phase = uld(&h->phase);
@@ -781,7 +792,7 @@ __device__ void run_query(const Ctx &c, u32 qs, bool retry, u32 lane, u32 *lut) 
         if (lane == 0) st_u64(c.cand + (u64)qs * c.WR, mk_key(d, c.entry));
         __syncwarp();
       } else {
-        if (!issue_batch(c, qs, false, lane)) return;
+        if (!issue_batch(c, qs, lane)) return;
       }
     } else if (phase == PH_EVAL) {
       const u32 nf = merge_select_dispatch(c, qs, lane);
@@ -798,7 +809,7 @@ __device__ void run_query(const Ctx &c, u32 qs, bool retry, u32 lane, u32 *lut) 
         if (it > c.max_iters) raise(c, 6, 0xA1, qs, it);
       }
       __syncwarp();
-      if (!issue_batch(c, qs, false, lane)) return;
+      if (!issue_batch(c, qs, lane)) return;
     } else {  // PH_EXPAND complete
       const u32 nf = uld(&h->n_items);
       const u32 nn = collect_neighbors(c, qs, lane);
@@ -816,7 +827,7 @@ __device__ void run_query(const Ctx &c, u32 qs, bool retry, u32 lane, u32 *lut) 
       if (lane == 0) { st_u32(&h->n_items, nn); st_u32(&h->phase, PH_EVAL); }
       __syncwarp();
       if (!PQ && nn > 0) {
-        if (!issue_batch(c, qs, false, lane)) return;
+        if (!issue_batch(c, qs, lane)) return;
       }
     }
   }
@@ -863,8 +874,13 @@ __global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
     if (warp_stopped(c)) break;
     u32 v;
     if (warp_pop(c, c.arr, v, lane)) { consume_arrival(c, v, lane); idle = 0; continue; }
-    if (warp_pop(c, c.run, v, lane)) { run_query<PQ>(c, v, false, lane, lut); idle = 0; continue; }
-    if (warp_pop(c, c.retry, v, lane)) { run_query<PQ>(c, v, true, lane, lut); idle = 0; __nanosleep(200); continue; }
+    if (warp_pop(c, c.run, v, lane)) { run_query<PQ>(c, v, lane, lut); idle = 0; continue; }
+    // nothing to run: see whether a page waiting for a slot can be given one
+    if (lane == 0 && (int)ld_u32((const u32 *)c.want.count) > 0) {
+      LaneStats st = {0, 0, 0, 0, 0, 0};
+      serve_want(c, kNil, st);
+      stat_add(c, S_EVICT, st.evict); stat_add(c, S_POSTED, st.posted);
+    }
     ++idle;
     __nanosleep(idle < 16 ? 100 : 1000);
     u32 late = ((idle & 127u) == 0 && globaltimer() - t0 > c.timeout_ns) ? 1u : 0u;
@@ -879,30 +895,30 @@ __global__ void init_kernel(const Ctx c) {
   const u32 tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
   for (u32 i = tid; i < c.n_qslots; i += nth) reset_hdr(c.hdr + i, i);
   // runnable queue starts with every slot; the others start empty
-  u64 *run = (u64 *)c.run.buf, *arr = (u64 *)c.arr.buf, *rty = (u64 *)c.retry.buf;
+  u64 *run = (u64 *)c.run.buf, *arr = (u64 *)c.arr.buf, *want = (u64 *)c.want.buf;
   for (u32 i = tid; i <= c.run.mask; i += nth) run[i] = i < c.n_qslots ? (((u64)(i + 1u) << 32) | i) : ((u64)i << 32);
-  for (u32 i = tid; i <= c.retry.mask; i += nth) rty[i] = (u64)i << 32;
   for (u32 i = tid; i <= c.arr.mask; i += nth) arr[i] = (u64)i << 32;
+  for (u32 i = tid; i <= c.want.mask; i += nth) want[i] = (u64)i << 32;
   if (tid == 0) {
     Ctl *ctl = c.ctl;
     ctl->stop = 0; ctl->status = 0; ctl->next_query = c.n_qslots; ctl->done = 0; ctl->ring_head = 0;
-    for (int i = 0; i < 8; ++i) { ctl->q_heads[i] = 0; ctl->dbg[i] = 0; }
+    for (int i = 0; i < 12; ++i) ctl->q_heads[i] = 0;
+    for (int i = 0; i < 8; ++i) ctl->dbg[i] = 0;
     *c.run.tail = c.n_qslots;
+    *c.run.count = (int)c.n_qslots;
   }
 }
 
-// Empty the cache; slots 0..preloaded-1 are marked READY holding pages 0..preloaded-1
-// (their bytes were copied there by the host before this kernel).
+// Empty the cache; slots 0..preloaded-1 hold pages 0..preloaded-1 (their bytes were copied
+// there by the host before this kernel) and are RESIDENT.
 __global__ void cache_reset_kernel(const Ctx c, u32 preloaded) {
   const u32 tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
-  const u32 n_tags = c.n_sets * kWays;
-  for (u32 ti = tid; ti < n_tags; ti += nth) {
-    const u32 slot = (ti % kWays) * c.n_sets + ti / kWays;
-    const bool pre = slot < preloaded;     // page p preloads into slot p: set p % n_sets, way p / n_sets
-    c.tag[ti] = pre ? mk_tag(slot, 1, 1, ST_READY) : mk_tag(kInvalidId, 0, 0, ST_EMPTY);
-    c.wl[ti] = pre ? ((1ull << 32) | kClosed) : (u64)kClosed;
+  for (u32 p = tid; p < c.n_pages; p += nth) c.ptab[p] = p < preloaded ? mk_pw(P_RESIDENT, p, 1) : kAbsentWord;
+  for (u32 s = tid; s < c.n_slots; s += nth) {
+    c.smeta[s] = s < preloaded ? mk_sm(s, 1, 1) : mk_sm(kInvalidId, 0, 0);
+    c.parts[s] = 0;
   }
-  for (u32 s = tid; s < c.n_sets; s += nth) c.hand[s] = 0;
+  if (tid == 0) { c.cs->bump = preloaded; c.cs->hand = 0; }
 }
 
 // Proxy copy batch: block b copies page b of the batch from host-mapped memory into its
