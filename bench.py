@@ -219,7 +219,7 @@ def main():
     ms = statistics.mean(times)
     st = stats_list[len(stats_list) // 2]
     fetched = statistics.mean(s["pages_fetched"] for s in stats_list)
-    launches = sum(2 + s["proxy_batches"] for s in stats_list)
+    launches = 2 * len(stats_list)          # init + persistent search kernel per step
 
     # roofline: the slowest of (a) algorithmic HBM bytes at the measured copy peak, (b) fetched
     # page bytes over the measured host link, (c) outstanding window / injected latency
@@ -260,7 +260,10 @@ def main():
                      "pages_fetched": fetched, "algorithmic_hbm_bytes": b_hbm,
                      "hbm_achieved_gbs": b_hbm / (ms * 1e-3) / 1e9, "hbm_peak_gbs": pk["hbm_gbs"]},
         "stats": {k: st[k] for k in ("pages_hit", "pages_missed", "pages_fetched", "dedupe_joins", "evictions",
-                                     "retries", "max_outstanding_seen", "resumes", "proxy_batches")},
+                                     "retries", "max_outstanding_seen", "resumes", "proxy_batches", "proxy_service_ns",
+                                     "proxy_iters", "proxy_ack_wait_iters", "proxy_window_full_iters",
+                                     "proxy_ring_empty_iters", "proxy_outstanding_sum", "warp_ns_arrivals",
+                                     "warp_ns_queries", "warp_ns_idle", "arrivals_consumed")},
     }
     if rank == 0 and world == 1:
         v, n_s = oracle_qps(w, threads)

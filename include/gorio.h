@@ -75,18 +75,18 @@ typedef struct {
  * Page cache + remote tier configuration (Section 3.2: GPU page-cache slots with one
  * ready entry each; Section 3.3: the proxy "batches submissions and completions,
  * controls outstanding remote I/O").
- *   capacity_pages   HBM cache size in 4 KB slots.  The cache is a 16-way set-associative
- *                    lock-free hash with a clock hand per set; capacity is rounded down
- *                    to a multiple of 16, except that capacity >= n_pages makes every
- *                    page resident-capable.  Must be >= 16.
+ *   capacity_pages   HBM cache size in 4 KB slots (>= 16; capped at the number of pages).
+ *                    Pages map to slots through a lock-free table with one state word per
+ *                    page; victims are chosen by a clock hand with reference bits.
  *   remote_latency_ns  a request's completion is published no earlier than this long
  *                    after the proxy admitted it.
  *   max_outstanding  most requests admitted and not yet published (>= 1).
  *   preload          1: fill the cache with pages 0..capacity-1 now (whole index when
  *                    capacity >= n_pages); 0: start cold.
  *   timeout_ms       bound on one gorio_search call (device and host waits); 0 = 60000.
- *   fill_batch       pages per proxy copy batch (1..128), 0 = default.  The proxy moves
- *                    pages with batched gather-copy kernels enqueued on its own streams.
+ * The proxy moves a page by writing a copy command into host-mapped memory; warps of the
+ * search kernel pull the page from the pinned store into its slot and acknowledge, and the
+ * proxy publishes the completion after the latency.  No CUDA call is made while a search runs.
  * Calling it again re-creates an empty (or preloaded) cache.
  */
 typedef struct {
@@ -95,8 +95,8 @@ typedef struct {
   uint32_t max_outstanding;
   uint32_t preload;
   uint32_t timeout_ms;
-  uint32_t fill_batch;
-  uint32_t reserved;
+  uint32_t reserved0;
+  uint32_t reserved1;
 } gorio_cache_cfg;
 
 /*
@@ -119,8 +119,8 @@ typedef struct {
  *   pages_missed   (query, node) waits registered on a page in flight (owner or joiner)
  *   pages_fetched  request descriptors the proxy serviced (4 KB each)
  *   dedupe_joins   waits that joined another query's or lane's outstanding request
- *   evictions, retries (lookups deferred because the set had no evictable slot or a
- *   validation failed), max_outstanding_seen (proxy), queries_done,
+ *   evictions, retries (hits that were evicted under the read and looked up again),
+ *   max_outstanding_seen (proxy), queries_done,
  *   n_eval / n_expand / sum_degree: totals of the per-query search counters (used for
  *   the algorithmic byte count), search_ns: wall time of the blocking search calls.
  * Hit/miss/fetch counts depend on timing; they obey invariants, not fixed values.
@@ -129,7 +129,17 @@ typedef struct {
   uint64_t pages_hit, pages_missed, pages_fetched;
   uint64_t dedupe_joins, evictions, retries, max_outstanding_seen, queries_done;
   uint64_t n_eval, n_expand, sum_degree, n_iter;
-  uint64_t resumes, search_ns, proxy_batches, reserved0;
+  uint64_t resumes, search_ns, proxy_batches, posted;
+  /* proxy diagnostics: sum over published requests of (publish - admit) in ns; loop
+     iterations in total / that found the head copy not yet acknowledged / with the window
+     full and a descriptor waiting / with room in the window but no descriptor; sum over
+     iterations of the requests in service (divide by proxy_iters for the time average) */
+  uint64_t proxy_service_ns, proxy_iters, proxy_ack_wait_iters, proxy_window_full_iters;
+  uint64_t proxy_ring_empty_iters, proxy_outstanding_sum;
+  /* where the worker warps' time went, ns summed over warps: serving arrived pages,
+     running query phases, idle; and the number of arrival-queue items consumed */
+  uint64_t warp_ns_arrivals, warp_ns_queries, warp_ns_idle, arrivals_consumed;
+  uint64_t reserved1, reserved2;
 } gorio_stats_t;
 
 /* Open an index on CUDA device `cuda_device`.  *out is set only on GORIO_OK. */

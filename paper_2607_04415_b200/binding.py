@@ -37,8 +37,8 @@ class _IndexDesc(ctypes.Structure):
 class _CacheCfg(ctypes.Structure):
     _fields_ = [("capacity_pages", ctypes.c_uint64), ("remote_latency_ns", ctypes.c_uint32),
                 ("max_outstanding", ctypes.c_uint32), ("preload", ctypes.c_uint32),
-                ("timeout_ms", ctypes.c_uint32), ("fill_batch", ctypes.c_uint32),
-                ("reserved", ctypes.c_uint32)]
+                ("timeout_ms", ctypes.c_uint32), ("reserved0", ctypes.c_uint32),
+                ("reserved1", ctypes.c_uint32)]
 
 
 class _Tuning(ctypes.Structure):
@@ -48,7 +48,10 @@ class _Tuning(ctypes.Structure):
 
 _STAT_FIELDS = ["pages_hit", "pages_missed", "pages_fetched", "dedupe_joins", "evictions", "retries",
                 "max_outstanding_seen", "queries_done", "n_eval", "n_expand", "sum_degree", "n_iter",
-                "resumes", "search_ns", "proxy_batches", "reserved0"]
+                "resumes", "search_ns", "proxy_batches", "posted", "proxy_service_ns", "proxy_iters",
+                "proxy_ack_wait_iters", "proxy_window_full_iters", "proxy_ring_empty_iters",
+                "proxy_outstanding_sum", "warp_ns_arrivals", "warp_ns_queries", "warp_ns_idle",
+                "arrivals_consumed", "reserved1", "reserved2"]
 
 
 class Stats(ctypes.Structure):
@@ -128,9 +131,9 @@ class Index:
             raise GorioError(status, detail or self._lib.gorio_status_str(status).decode())
 
     def cache_config(self, capacity_pages, remote_latency_ns=0, max_outstanding=256, preload=False,
-                     timeout_ms=0, fill_batch=0):
+                     timeout_ms=0):
         cfg = _CacheCfg(int(capacity_pages), int(remote_latency_ns), int(max_outstanding), int(bool(preload)),
-                        int(timeout_ms), int(fill_batch), 0)
+                        int(timeout_ms), 0, 0)
         self._check(self._lib.gorio_cache_config(self._h, ctypes.byref(cfg)))
 
     def set_tuning(self, max_inflight=0, visited_capacity=0, warps_per_block=0, blocks_per_sm=0):

@@ -6,6 +6,7 @@
 #include <chrono>
 #include <condition_variable>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <deque>
 #include <mutex>
@@ -21,7 +22,6 @@ using namespace gorio;
 
 namespace {
 
-constexpr int kMaxFillStreams = 4;
 typedef std::chrono::steady_clock Clock;
 
 inline u32 next_pow2(u64 v) { u32 p = 1; while (p < v) p <<= 1; return p; }
@@ -48,11 +48,13 @@ struct gorio_index {
   u32 *parts = nullptr;
   CacheShared *cs = nullptr;
   u64 *want_buf = nullptr; u32 want_cap = 0;
+  u64 *cpy_buf = nullptr, *fcmd_mirror = nullptr;
   // host-mapped communication areas
   u64 *ring_h = nullptr; u64 *ring_d = nullptr; u32 ring_cap = 0;
   u32 *comp_h = nullptr; u32 *comp_d = nullptr;
-  u32 *hctl_h = nullptr; u32 *hctl_d = nullptr;     // [0] completion tail, [1] abort, [8..] copied flags
-  u32 *fill_counters = nullptr;                     // device, one per fill stream
+  u32 *hctl_h = nullptr; u32 *hctl_d = nullptr;     // [0] completion tail, [1] abort, [2] copy-command tail
+  u64 *fcmd_h = nullptr; u64 *fcmd_d = nullptr;     // copy commands, proxy -> GPU
+  u32 *fdone_h = nullptr; u32 *fdone_d = nullptr;   // copy acknowledgements, GPU -> proxy
   u64 *arr_buf = nullptr; u32 arr_cap = 0;
 
   // query state
@@ -75,12 +77,12 @@ struct gorio_index {
   std::atomic<int> px_stop{0};
   std::atomic<int> px_active{0};
   std::atomic<int> px_error{0};
-  cudaStream_t fill_streams[kMaxFillStreams] = {};
   cudaStream_t own_stream = nullptr;
   cudaEvent_t done_ev = nullptr;
 
   // statistics
   u64 host_fetched = 0, host_max_out = 0, host_batches = 0, host_search_ns = 0;
+  u64 host_service_ns = 0, host_ack_wait = 0, host_window_full = 0, host_ring_empty = 0, host_iters = 0, host_out_sum = 0;
   u32 px_dbg[8] = {};   // proxy progress at the end of its last service loop
   std::string err;
 };
@@ -116,12 +118,16 @@ cudaError_t host_mapped(T **h, T **d, size_t count) {
 
 void free_cache(gorio_index *ix) {
   cudaFree(ix->slot_data); cudaFree(ix->ptab); cudaFree(ix->smeta); cudaFree(ix->parts); cudaFree(ix->cs);
-  cudaFree(ix->want_buf); cudaFree(ix->fill_counters);
+  cudaFree(ix->want_buf); cudaFree(ix->cpy_buf); cudaFree(ix->fcmd_mirror);
+  ix->cpy_buf = ix->fcmd_mirror = nullptr;
   if (ix->ring_h) cudaFreeHost(ix->ring_h);
   if (ix->comp_h) cudaFreeHost(ix->comp_h);
+  if (ix->fcmd_h) cudaFreeHost(ix->fcmd_h);
+  if (ix->fdone_h) cudaFreeHost(ix->fdone_h);
+  ix->fcmd_h = ix->fcmd_d = nullptr; ix->fdone_h = ix->fdone_d = nullptr;
   ix->slot_data = nullptr; ix->ptab = ix->smeta = nullptr; ix->parts = nullptr; ix->cs = nullptr;
   ix->want_buf = nullptr;
-  ix->fill_counters = nullptr; ix->ring_h = ix->ring_d = nullptr; ix->comp_h = ix->comp_d = nullptr;
+  ix->ring_h = ix->ring_d = nullptr; ix->comp_h = ix->comp_d = nullptr;
   ix->cache_ready = false;
 }
 
@@ -131,71 +137,68 @@ void free_qstate(gorio_index *ix) {
 }
 
 // ---------------------------------------------------------------------------------------
-// the proxy: consumes request descriptors in order, bounds the number in service, moves
-// page bytes from pinned host memory into cache slots, and publishes completions no
-// earlier than admission + latency.
+// the proxy: consumes request descriptors in order, bounds the number in service, commands
+// the copy of each page from pinned host memory into its cache slot, and publishes the
+// completion once the copy is acknowledged and no earlier than admission + latency.
+// It issues no CUDA calls while a search runs: commands, acknowledgements and completions
+// all travel through host-mapped memory.
 // ---------------------------------------------------------------------------------------
-struct InService { u32 slot; u32 stream; u32 seq; Clock::time_point admitted; };
+struct InService { u32 slot; u32 idx; Clock::time_point admitted; };
 
 void proxy_service(gorio_index *ix) {
   const u32 ring_mask = ix->ring_cap - 1, ring_shift = ilog2(ix->ring_cap);
   const u32 max_out = ix->cfg.max_outstanding;
-  const u32 batch_max = ix->cfg.fill_batch;
   const auto latency = std::chrono::nanoseconds(ix->cfg.remote_latency_ns);
-  const int n_streams = kMaxFillStreams;
   volatile u64 *ring = ix->ring_h;
-  volatile u32 *copied = ix->hctl_h + 8;
+  volatile u64 *fcmd = ix->fcmd_h;
+  volatile u32 *fdone = ix->fdone_h;
   u32 tail = 0, ct = 0, outstanding = 0;
-  u32 stream_seq[kMaxFillStreams] = {0, 0, 0, 0};
-  int k = 0;
   std::deque<InService> inflight;
-  FillBatch batch;
   u64 fetched = 0, max_seen = 0, batches = 0;
+  u64 service_ns = 0, ack_wait_iters = 0, window_full_iters = 0, ring_empty_iters = 0, iters = 0, out_sum = 0;
 
   while (!ix->px_stop.load(std::memory_order_acquire)) {
-    // 1. admit descriptors while the in-service window has room
-    batch.n = 0;
+    ++iters;
+    out_sum += outstanding;
+    // 1. admit descriptors while the in-service window has room; each becomes a copy command
+    u32 admitted = 0;
     const Clock::time_point now0 = Clock::now();
-    while (outstanding < max_out && batch.n < batch_max) {
+    while (outstanding < max_out) {
       const u64 e = ring[tail & ring_mask];
       const u32 lap = ((tail >> ring_shift) % 255u) + 1u;
       if ((u32)(e & 0xFFu) != lap) break;
-      std::atomic_thread_fence(std::memory_order_acquire);
-      batch.page[batch.n] = (u32)(e >> 32);
-      batch.slot[batch.n] = (u32)(e >> 8) & 0xFFFFFFu;
-      if (batch.page[batch.n] >= ix->n_pages || batch.slot[batch.n] >= ix->n_slots) {
+      const u32 page = (u32)(e >> 32), slot = (u32)(e >> 8) & 0xFFFFFFu;
+      if (page >= ix->n_pages || slot >= ix->n_slots) {
         ix->px_error.store(1);   // a descriptor the GPU could not have produced
         return;
       }
-      ++batch.n; ++tail; ++outstanding;
+      fcmd[tail & ring_mask] = e;                 // same index, same lap tag
+      inflight.push_back({slot, tail, now0});
+      ++tail; ++outstanding; ++admitted;
     }
-    if (batch.n) {
-      const u32 seq = ++stream_seq[k];
-      batch.seq = seq;
-      cudaError_t e = cudaSuccess;
-      e = launch_fill(batch, ix->pages_dev, ix->slot_data, ix->fill_counters + k,
-                      ix->hctl_d + 8 + k, ix->fill_streams[k]);
-      if (e != cudaSuccess) { ix->px_error.store(2); return; }
-      for (u32 i = 0; i < batch.n; ++i) inflight.push_back({batch.slot[i], (u32)k, seq, now0});
-      k = (k + 1) % n_streams;
+    if (admitted) {
       ++batches;
       if (outstanding > max_seen) max_seen = outstanding;
     }
-    // 2. publish completions in admission order: copy landed and latency elapsed
+    if (outstanding >= max_out) {
+      if ((u32)(ring[tail & ring_mask] & 0xFFu) == ((tail >> ring_shift) % 255u) + 1u) ++window_full_iters;
+    } else {
+      ++ring_empty_iters;
+    }
+    // 2. publish completions in admission order: copy acknowledged and latency elapsed
     if (!inflight.empty()) {
       const Clock::time_point now = Clock::now();
       u32 published = 0;
       while (!inflight.empty()) {
         const InService &r = inflight.front();
         if (now - r.admitted < latency) break;
-        if ((int)(copied[r.stream] - r.seq) < 0) break;
-        ix->comp_h[ct & ring_mask] = r.slot;
+        if (fdone[r.idx & ring_mask] != ((r.idx >> ring_shift) % 255u) + 1u) { ++ack_wait_iters; break; }
+        service_ns += (u64)std::chrono::duration_cast<std::chrono::nanoseconds>(now - r.admitted).count();
+        ix->comp_h[ct & ring_mask] = (r.slot << 8) | (((ct >> ring_shift) % 255u) + 1u);
         ++ct; ++published;
         inflight.pop_front();
       }
       if (published) {
-        std::atomic_thread_fence(std::memory_order_release);
-        ((volatile u32 *)ix->hctl_h)[0] = ct;
         outstanding -= published;
         fetched += published;
       }
@@ -203,9 +206,11 @@ void proxy_service(gorio_index *ix) {
   }
   ix->px_dbg[0] = tail; ix->px_dbg[1] = ct; ix->px_dbg[2] = outstanding; ix->px_dbg[3] = (u32)inflight.size();
   if (!inflight.empty()) {
-    ix->px_dbg[4] = inflight.front().stream; ix->px_dbg[5] = inflight.front().seq;
-    ix->px_dbg[6] = copied[inflight.front().stream];
+    ix->px_dbg[4] = inflight.front().idx;
+    ix->px_dbg[5] = fdone[inflight.front().idx & ring_mask];
   }
+  ix->host_service_ns += service_ns; ix->host_ack_wait += ack_wait_iters; ix->host_window_full += window_full_iters;
+  ix->host_ring_empty += ring_empty_iters; ix->host_iters += iters; ix->host_out_sum += out_sum;
   ix->host_fetched += fetched;
   ix->host_batches += batches;
   if (max_seen > ix->host_max_out) ix->host_max_out = max_seen;
@@ -261,20 +266,12 @@ int setup_cache(gorio_index *ix) {
   CK(cudaMalloc(&ix->parts, (size_t)ix->n_slots * 4));
   CK(cudaMalloc(&ix->cs, sizeof(CacheShared)));
   CK(cudaMalloc(&ix->want_buf, (size_t)ix->want_cap * 8));
-  CK(cudaMalloc(&ix->fill_counters, kMaxFillStreams * 4));
-  CK(cudaMemset(ix->fill_counters, 0, kMaxFillStreams * 4));
+  CK(cudaMalloc(&ix->cpy_buf, (size_t)ix->ring_cap * 8));
+  CK(cudaMalloc(&ix->fcmd_mirror, (size_t)ix->ring_cap * 8));
   CK(host_mapped(&ix->ring_h, &ix->ring_d, ix->ring_cap));
   CK(host_mapped(&ix->comp_h, &ix->comp_d, ix->ring_cap));
-  // Warm the whole proxy copy path (kernel code, launch path of every copy stream) before a
-  // persistent kernel can depend on it: copy page 0 into slot 0 once per stream.
-  {
-    FillBatch wb{};
-    wb.n = 1; wb.seq = 0; wb.page[0] = 0; wb.slot[0] = 0;
-    for (int i = 0; i < kMaxFillStreams; ++i) {
-      CK(launch_fill(wb, ix->pages_dev, ix->slot_data, ix->fill_counters + i, ix->hctl_d + 8 + i, ix->fill_streams[i]));
-      CK(cudaStreamSynchronize(ix->fill_streams[i]));
-    }
-  }
+  CK(host_mapped(&ix->fcmd_h, &ix->fcmd_d, ix->ring_cap));
+  CK(host_mapped(&ix->fdone_h, &ix->fdone_d, ix->ring_cap));
   ix->preloaded = 0;
   if (cfg.preload) {
     ix->preloaded = cap >= ix->n_pages ? ix->n_pages : ix->n_slots;
@@ -395,11 +392,6 @@ int gorio_index_open(const gorio_index_desc *d, int cuda_device, gorio_index **o
   if (host_mapped(&ix->hctl_h, &ix->hctl_d, 64) != cudaSuccess) return bail(GORIO_ERR_CUDA);
   if (cudaMalloc(&ix->ctl, sizeof(Ctl)) != cudaSuccess) return bail(GORIO_ERR_NOMEM);
   cudaMemset(ix->ctl, 0, sizeof(Ctl));
-  int lo = 0, hi = 0;
-  cudaDeviceGetStreamPriorityRange(&lo, &hi);
-  for (int i = 0; i < kMaxFillStreams; ++i)
-    if (cudaStreamCreateWithPriority(&ix->fill_streams[i], cudaStreamNonBlocking, hi) != cudaSuccess)
-      return bail(GORIO_ERR_CUDA);
   if (cudaStreamCreateWithFlags(&ix->own_stream, cudaStreamNonBlocking) != cudaSuccess) return bail(GORIO_ERR_CUDA);
   if (cudaEventCreateWithFlags(&ix->done_ev, cudaEventDisableTiming) != cudaSuccess) return bail(GORIO_ERR_CUDA);
   ix->proxy = std::thread(proxy_main, ix);
@@ -425,7 +417,6 @@ int gorio_index_close(gorio_index *ix) {
   cudaFree(ix->ctl);
   cudaFree(ix->st_q); cudaFree(ix->st_out);
   if (ix->hctl_h) cudaFreeHost(ix->hctl_h);
-  for (int i = 0; i < kMaxFillStreams; ++i) if (ix->fill_streams[i]) cudaStreamDestroy(ix->fill_streams[i]);
   if (ix->own_stream) cudaStreamDestroy(ix->own_stream);
   if (ix->done_ev) cudaEventDestroy(ix->done_ev);
   if (ix->registered_pages) cudaHostUnregister((void *)ix->desc.host_pages);
@@ -435,14 +426,13 @@ int gorio_index_close(gorio_index *ix) {
 
 int gorio_cache_config(gorio_index *ix, const gorio_cache_cfg *cfg) {
   if (!ix || !cfg) return GORIO_ERR_INVALID_ARG;
-  if (cfg->capacity_pages < 16 || cfg->max_outstanding < 1 || cfg->fill_batch > kMaxFillBatch)
-    return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: capacity >= 16, max_outstanding >= 1, fill_batch <= 128");
+  if (cfg->capacity_pages < 16 || cfg->max_outstanding < 1)
+    return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: capacity >= 16, max_outstanding >= 1");
   u64 cap = cfg->capacity_pages < ix->n_pages ? cfg->capacity_pages : ix->n_pages;
   if (cap >= (1ull << 24)) return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: at most 2^24 slots");
   CK(cudaSetDevice(ix->dev));
   ix->cfg = *cfg;
   if (ix->cfg.timeout_ms == 0) ix->cfg.timeout_ms = 60000;
-  if (ix->cfg.fill_batch == 0) ix->cfg.fill_batch = 128;
   return setup_cache(ix);
 }
 
@@ -482,22 +472,27 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   c.n_slots = ix->n_slots;
   c.ring = ix->ring_d; c.ring_mask = ix->ring_cap - 1; c.ring_shift = ilog2(ix->ring_cap);
   c.comp_ring = ix->comp_d; c.comp_mask = ix->ring_cap - 1; c.host_ctl = ix->hctl_d;
+  c.fcmd = ix->fcmd_d; c.fdone = ix->fdone_d; c.host_pages = ix->pages_dev;
   c.ctl = ix->ctl;
   u32 *qh = ix->ctl->q_heads;
   c.arr = Queue{(u32 *)ix->arr_buf, ix->arr_cap - 1, qh + 0, qh + 1, (int *)(qh + 2)};
   c.run = Queue{(u32 *)ix->run_buf, ix->runq_cap - 1, qh + 3, qh + 4, (int *)(qh + 5)};
   c.want = Queue{(u32 *)ix->want_buf, ix->want_cap - 1, qh + 6, qh + 7, (int *)(qh + 8)};
+  c.cpy = Queue{(u32 *)ix->cpy_buf, ix->ring_cap - 1, qh + 9, qh + 10, (int *)(qh + 11)};
+  c.fcmd_dev = ix->fcmd_mirror;
   c.nq = nq; c.K = K; c.L = L; c.W = W; c.WR = ix->qs_WR;
   c.queries = queries_dev; c.out_ids = out_ids_dev; c.out_dists = out_dists_dev;
   c.out_pages = out_pages_distinct_dev; c.out_counters = out_counters_dev;
   c.timeout_ns = (u64)ix->cfg.timeout_ms * 1000000ull;
   c.max_iters = 64u * L + 1024u;
+  { const char *e = std::getenv("GORIO_CENSUS_MS"); c.census_ns = e ? (u64)std::atof(e) * 1000000ull : 0; }
 
   // launch geometry: leave room on every SM for the proxy's copy kernels
   const bool pq = d.pq_m != 0;
-  u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 6u : 16u);
+  // warps per block = worker warps + one copier warp (block 0 also hosts the completion poller)
+  u32 warps = (ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 5u : 16u)) + 1u;
   if (pq) { u32 lim = (200u * 1024u) / (d.pq_m * kPqKsub * 4u); if (warps > lim) warps = lim; }
-  if (warps < 2) return fail(ix, GORIO_ERR_INVALID_ARG, "search: shared memory cannot hold two PQ tables per block");
+  if (warps < 3) return fail(ix, GORIO_ERR_INVALID_ARG, "search: shared memory cannot hold the PQ tables of a block");
   int occ = 0;
   CK(search_occupancy(d.pq_m, warps, &occ));
   if (occ < 1) return fail(ix, GORIO_ERR_INVALID_ARG, "search: launch geometry does not fit an SM");
@@ -507,6 +502,9 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
 
   // reset the host-visible rings while the proxy is idle
   std::memset(ix->ring_h, 0, (size_t)ix->ring_cap * 8);
+  std::memset(ix->fcmd_h, 0, (size_t)ix->ring_cap * 8);
+  std::memset(ix->fdone_h, 0, (size_t)ix->ring_cap * 4);
+  std::memset(ix->comp_h, 0, (size_t)ix->ring_cap * 4);
   std::memset(ix->hctl_h, 0, 64 * 4);
   std::atomic_thread_fence(std::memory_order_seq_cst);
 
@@ -529,23 +527,27 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
     std::this_thread::sleep_for(std::chrono::microseconds(20));
   }
   proxy_stop(ix);
-  for (int i = 0; i < kMaxFillStreams; ++i) cudaStreamSynchronize(ix->fill_streams[i]);
   if (qe != cudaSuccess) return cuda_fail(ix, qe, "search kernel");
   Ctl h{};
   CK(cudaMemcpyAsync(&h, ix->ctl, sizeof(Ctl), cudaMemcpyDeviceToHost, stream));
   CK(cudaStreamSynchronize(stream));
   ix->host_search_ns += (u64)std::chrono::duration_cast<std::chrono::nanoseconds>(Clock::now() - t_begin).count();
-  if (ix->px_error.load()) return fail(ix, GORIO_ERR_INTERNAL, "proxy: bad descriptor or copy launch failure");
+  if (c.census_ns)
+    std::fprintf(stderr, "[gorio census] slots: unused %u, changing owner %u, FILLING %u, ARRIVED %u, RESIDENT ref %u, RESIDENT noref %u | "
+                 "pages WANTED %u | queries awaiting %u (items %u) | queues want %d arr %d run %d | done %u posted %u\n",
+                 h.census[0], h.census[1], h.census[2], h.census[3], h.census[4], h.census[5], h.census[6], h.census[7],
+                 h.census[8], (int)h.census[9], (int)h.census[10], (int)h.census[11], h.census[12], h.census[13]);
+  if (ix->px_error.load()) return fail(ix, GORIO_ERR_INTERNAL, "proxy: descriptor out of range");
   if (h.status != 0 || h.stop != 1) {
     char buf[640];
     const u32 s = h.status ? h.status : (u32)GORIO_ERR_INTERNAL;
     std::snprintf(buf, sizeof buf,
                   "device: %s (site 0x%x, %u, %u, %u; block %u thread %u; done %u/%u; posted %u; arrivals %u/%u; "
                   "runnable %u/%u; want %u/%u; proxy consumed %u published %u outstanding %u queued %u "
-                  "[head stream %u seq %u copied %u])",
+                  "[head command %u ack %u])",
                   s < 9 ? kDeviceErr[s] : "?", h.dbg[0], h.dbg[1], h.dbg[2], h.dbg[3], h.dbg[4], h.dbg[5], h.done, nq,
                   h.ring_head, h.q_heads[0], h.q_heads[1], h.q_heads[3], h.q_heads[4], h.q_heads[6], h.q_heads[7],
-                  ix->px_dbg[0], ix->px_dbg[1], ix->px_dbg[2], ix->px_dbg[3], ix->px_dbg[4], ix->px_dbg[5], ix->px_dbg[6]);
+                  ix->px_dbg[0], ix->px_dbg[1], ix->px_dbg[2], ix->px_dbg[3], ix->px_dbg[4], ix->px_dbg[5]);
     return fail(ix, (int)s, buf);
   }
   ix->cache_dirty = false;
@@ -588,7 +590,12 @@ int gorio_stats(gorio_index *ix, gorio_stats_t *out) {
   out->max_outstanding_seen = ix->host_max_out; out->queries_done = h.stats[S_DONE];
   out->n_eval = h.stats[S_NEVAL]; out->n_expand = h.stats[S_NEXPAND]; out->sum_degree = h.stats[S_SUMDEG];
   out->n_iter = h.stats[S_NITER]; out->resumes = h.stats[S_RESUMES]; out->search_ns = ix->host_search_ns;
-  out->proxy_batches = ix->host_batches; out->reserved0 = h.stats[S_POSTED];
+  out->proxy_batches = ix->host_batches; out->posted = h.stats[S_POSTED];
+  out->proxy_service_ns = ix->host_service_ns; out->proxy_ack_wait_iters = ix->host_ack_wait;
+  out->proxy_window_full_iters = ix->host_window_full; out->proxy_ring_empty_iters = ix->host_ring_empty;
+  out->proxy_iters = ix->host_iters; out->proxy_outstanding_sum = ix->host_out_sum;
+  out->warp_ns_arrivals = h.stats[S_T_ARR]; out->warp_ns_queries = h.stats[S_T_RUN]; out->warp_ns_idle = h.stats[S_T_IDLE];
+  out->arrivals_consumed = h.stats[S_N_ARR];
   return GORIO_OK;
 }
 
@@ -597,6 +604,7 @@ int gorio_stats_reset(gorio_index *ix) {
   CK(cudaSetDevice(ix->dev));
   CK(cudaMemset((u8 *)ix->ctl + offsetof(Ctl, stats), 0, sizeof(((Ctl *)0)->stats)));
   ix->host_fetched = ix->host_max_out = ix->host_batches = ix->host_search_ns = 0;
+  ix->host_service_ns = ix->host_ack_wait = ix->host_window_full = ix->host_ring_empty = ix->host_iters = ix->host_out_sum = 0;
   return GORIO_OK;
 }
 

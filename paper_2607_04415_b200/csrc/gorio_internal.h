@@ -16,7 +16,6 @@ constexpr u32 kNil = 0xFFFFFFFFu;     // end of a waiter list
 constexpr u32 kClosed = 0xFFFFFFFEu;  // waiter list closed: the page has arrived
 constexpr u32 kInvalidId = 0xFFFFFFFFu;
 constexpr u64 kPadKey = ~0ull;        // sorts after every real key
-constexpr u32 kMaxFillBatch = 128;
 constexpr u32 kPqKsub = 256;
 
 // Query phases: which batch of page items is outstanding for the query slot.
@@ -58,13 +57,14 @@ struct Ctl {
   u32 next_query;  // next query id to admit when a slot frees
   u32 done;        // queries finished
   u32 ring_head;   // request descriptors posted
-  u32 q_heads[12]; // queue head/tail/count words: arr(0,1,2) run(3,4,5) want(6,7,8)
+  u32 q_heads[16]; // queue head/tail/count words: arr(0,1,2) run(3,4,5) want(6,7,8) copy(9,10,11)
   u32 dbg[8];      // detail of the first error
+  u32 census[16];  // debug snapshot (see census())
   u64 stats[16];
 };
 
 enum StatIdx { S_HIT = 0, S_MISSED, S_JOINS, S_EVICT, S_RETRY, S_DONE, S_NEVAL, S_NEXPAND,
-               S_SUMDEG, S_NITER, S_RESUMES, S_POSTED };
+               S_SUMDEG, S_NITER, S_RESUMES, S_POSTED, S_T_ARR, S_T_RUN, S_T_IDLE, S_N_ARR };
 
 // Everything the persistent kernel needs, passed by value.
 struct Ctx {
@@ -83,10 +83,15 @@ struct Ctx {
   // miss ring: host-mapped, written by the GPU, consumed by the proxy
   u64 *ring;
   u32 ring_mask, ring_shift;
-  // completions: host-mapped, written by the proxy, polled by the GPU
-  const u32 *comp_ring;
+  // completions and copy commands: host-mapped, written by the proxy, read by the GPU
+  const u32 *comp_ring; // completions [slot:24][lap:8]
   u32 comp_mask;
-  const u32 *host_ctl;  // [0] completion tail, [1] abort request
+  const u32 *host_ctl;  // [1] abort request
+  const u64 *fcmd;      // copy commands [page:32][slot:24][lap:8], same size as the miss ring
+  u32 *fdone;           // per-command acknowledgement (lap tag), written by the GPU
+  const u8 *host_pages; // device view of the pinned host page store
+  Queue cpy;              // indices of copy commands ready for the copier warps
+  u64 *fcmd_dev;          // device mirror of the copy-command ring
   Queue arr, run, want;   // arrivals (slots / chain continuations), runnable query slots, pages awaiting a slot
   // query state
   u32 n_qslots, nq, K, L, W, WR;
@@ -108,14 +113,8 @@ struct Ctx {
   u32 *out_counters;
   Ctl *ctl;
   u64 timeout_ns;
+  u64 census_ns;   // debug: take a state census this long after the kernel started (0 = never)
   u32 max_iters;
-};
-
-struct FillBatch {
-  u32 n;
-  u32 seq;
-  u32 page[kMaxFillBatch];
-  u32 slot[kMaxFillBatch];
 };
 
 // launchers implemented in search_kernels.cu
@@ -123,8 +122,6 @@ cudaError_t preload_kernels();
 cudaError_t launch_init(const Ctx &c, cudaStream_t s);
 cudaError_t launch_search(const Ctx &c, u32 blocks, u32 warps_per_block, cudaStream_t s);
 cudaError_t search_occupancy(u32 pq_m, u32 warps_per_block, int *blocks_per_sm);
-cudaError_t launch_fill(const FillBatch &b, const u8 *host_pages_dev, u8 *slot_data,
-                        u32 *counter, u32 *host_copied, cudaStream_t s);
 cudaError_t launch_cache_reset(const Ctx &c, u32 preloaded_pages, cudaStream_t s);
 
 }  // namespace gorio

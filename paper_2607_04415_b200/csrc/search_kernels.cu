@@ -46,6 +46,17 @@ __device__ __forceinline__ void st_u16(u16 *p, u16 v) {
 __device__ __forceinline__ u32 ld_sys_u32(const u32 *p) {
   u32 v; asm volatile("ld.relaxed.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory"); return v;
 }
+__device__ __forceinline__ u64 ld_sys_u64(const u64 *p) {
+  u64 v; asm volatile("ld.relaxed.sys.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory"); return v;
+}
+__device__ __forceinline__ uint4 ld_sys_v4(const u32 *p) {
+  uint4 v;
+  asm volatile("ld.volatile.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_sys_u32(u32 *p, u32 v) {
+  asm volatile("st.relaxed.sys.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 __device__ __forceinline__ void st_sys_u64(u64 *p, u64 v) {
   asm volatile("st.relaxed.sys.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
@@ -834,29 +845,172 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut) {
   if (lane == 0) raise(c, 6, 0xA2, qs);
 }
 
-// Warp 0 of block 0: forwards the proxy's completion ring (host memory) into the arrival
-// queue in HBM, watches the host's abort word and the deadline.
-__device__ void poller(const Ctx &c, u32 lane) {
-  u32 seen = 0, it = 0;
+// Copier warps (the last warp of every block) execute the proxy's copy commands, which the
+// poller mirrors into device memory: pull the 4 KB page from the pinned store into the cache
+// slot (each lane moves 8 x 16 bytes, all loads in flight before the first store) and
+// acknowledge to the host, which publishes the completion once the latency has elapsed.
+// Only the page bytes cross the host link on this path; no copier ever polls host memory.
+__device__ void copier(const Ctx &c, u32 lane) {
+  u32 idle = 0;
   const u64 t0 = globaltimer();
   for (;;) {
     if (warp_stopped(c)) break;
-    u32 tail = 0, abort_req = 0;
-    if (lane == 0) { tail = ld_sys_u32(c.host_ctl); abort_req = ld_sys_u32(c.host_ctl + 1); }
-    tail = __shfl_sync(0xffffffffu, tail, 0);
-    abort_req = __shfl_sync(0xffffffffu, abort_req, 0);
-    if (abort_req) { if (lane == 0) raise(c, 5, 0xB1); break; }
-    while (seen != tail) {
-      const u32 nn = min(32u, tail - seen);
-      if (lane < nn) {
-        u32 slot = ld_sys_u32(c.comp_ring + ((seen + lane) & c.comp_mask));
-        q_push(c, c.arr, slot);
-      }
-      seen += nn;
-      __syncwarp();
+    u32 idx;
+    if (!warp_pop(c, c.cpy, idx, lane)) {
+      ++idle;
+      __nanosleep(idle < 64 ? 100 : 1000);
+      u32 late = ((idle & 255u) == 0 && globaltimer() - t0 > c.timeout_ns) ? 1u : 0u;
+      if (__shfl_sync(0xffffffffu, late, 0)) { if (lane == 0) raise(c, 5, 0xB4); break; }
+      continue;
     }
-    u32 late = ((++it & 255u) == 0 && globaltimer() - t0 > c.timeout_ns) ? 1u : 0u;
-    if (__shfl_sync(0xffffffffu, late, 0)) { if (lane == 0) raise(c, 5, 0xB2); break; }
+    idle = 0;
+    const u64 cmd = __shfl_sync(0xffffffffu, ld_u64(c.fcmd_dev + (idx & c.ring_mask)), 0);
+    const u32 page = (u32)(cmd >> 32), slot = (u32)(cmd >> 8) & 0xFFFFFFu;
+    if (page >= c.n_pages || slot >= c.n_slots) { if (lane == 0) raise(c, 8, 0xC1, idx, page, slot); break; }
+    const uint4 *src = (const uint4 *)(c.host_pages + (u64)page * kPageBytes);
+    uint4 *dst = (uint4 *)(c.slot_data + (u64)slot * kPageBytes);
+    uint4 v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __ldcs(src + i * 32 + lane);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) __stcg(dst + i * 32 + lane, v[i]);
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) {
+      __threadfence_system();
+      st_sys_u32(c.fdone + (idx & c.ring_mask), (u32)cmd & 0xFFu);
+    }
+  }
+}
+
+// Push n values (lane-distributed: value k of this lane goes to position rank0 + k if
+// take[k]) with one ticket reservation and one count update for the whole warp.
+__device__ __forceinline__ void bulk_push4(const Ctx &c, const Queue &q, const u32 (&val)[4], const bool (&take)[4],
+                                           u32 n, u32 first_rank, u32 lane) {
+  if (n == 0) return;
+  u32 base = 0;
+  if (lane == 0) { __threadfence(); base = atomicAdd(q.tail, n); }
+  base = __shfl_sync(0xffffffffu, base, 0);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    if (take[k]) {
+      const u32 pos = base + first_rank + (u32)k;
+      u64 *cell = (u64 *)q.buf + (pos & q.mask);
+      u32 spins = 0;
+      while ((u32)(ld_u64(cell) >> 32) != pos) {
+        if (++spins > kSpinLimit) { raise(c, 8, 0x53, pos); break; }
+      }
+      st_u64(cell, ((u64)(pos + 1u) << 32) | val[k]);
+    }
+  }
+  __syncwarp();
+  if (lane == 0) atomicAdd(q.count, (int)n);
+}
+
+// Warp 0 of block 0 is the only warp that reads control data from host memory.  Per
+// iteration it reads the next 128 positions of the proxy's completion ring and of its
+// copy-command ring (both self-validating through a lap tag, one 512-byte read each, issued
+// together), forwards new completions to the arrival queue and new commands, mirrored
+// into device memory, to the copy queue.  The abort word is sampled now and then.
+__device__ void ring_window(const Ctx &c, const u32 (&e)[4], u32 base, u32 seen, u32 lane, u32 &end) {
+  u32 first_bad = 128;
+#pragma unroll
+  for (int k = 3; k >= 0; --k) {
+    const u32 i = base + 4u * lane + (u32)k;
+    const bool ok = (e[k] & 0xFFu) == ((i >> c.ring_shift) % 255u) + 1u || i < seen;
+    if (!ok) first_bad = 4u * lane + (u32)k;
+  }
+  end = base + __reduce_min_sync(0xffffffffu, first_bad);    // entries [seen, end) are new and valid
+}
+
+// Debug aid: one snapshot of where slots, pages and queries are, taken by the poller warp.
+__device__ void census(const Ctx &c, u32 lane) {
+  u32 cnt[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+  for (u32 s = lane; s < c.n_slots; s += 32) {
+    const u64 m = ld_u64(c.smeta + s);
+    const u32 pg = sm_page(m);
+    if (pg >= c.n_pages) { cnt[0]++; continue; }
+    const u64 w = ld_u64(c.ptab + pg);
+    if (pw_slot(w) != s || pw_state(w) < P_FILLING) { cnt[1]++; continue; }   // slot between owners
+    if (pw_state(w) == P_FILLING) cnt[2]++;
+    else if (pw_state(w) == P_ARRIVED) cnt[3]++;
+    else if (m & 1ull) cnt[4]++; else cnt[5]++;
+  }
+  for (u32 p = lane; p < c.n_pages; p += 32) {
+    const u32 st = pw_state(ld_u64(c.ptab + p));
+    if (st == P_WANTED) cnt[6]++;
+  }
+  for (u32 q = lane; q < c.n_qslots; q += 32) {
+    const u32 aw = ld_u32(&c.hdr[q].awaiting);
+    if (aw > 0) { cnt[7]++; cnt[8] += aw; }
+  }
+  for (int i = 0; i < 12; ++i) cnt[i] = __reduce_add_sync(0xffffffffu, cnt[i]);
+  if (lane == 0) {
+    for (int i = 0; i < 9; ++i) c.ctl->census[i] = cnt[i];
+    c.ctl->census[9] = (u32)*c.want.count; c.ctl->census[10] = (u32)*c.arr.count; c.ctl->census[11] = (u32)*c.run.count;
+    c.ctl->census[12] = ld_u32(&c.ctl->done); c.ctl->census[13] = ld_u32(&c.ctl->ring_head);
+  }
+}
+
+__device__ void poller(const Ctx &c, u32 lane) {
+  u32 seen = 0, seen_cmd = 0, it = 0;
+  const u64 t0 = globaltimer();
+  bool census_done = c.census_ns == 0;
+  for (;;) {
+    if (warp_stopped(c)) break;
+    if (!census_done && globaltimer() - t0 > c.census_ns) { census(c, lane); census_done = true; }
+    const u32 base = seen & ~3u, cbase = seen_cmd & ~1u;
+    // completions: 4 x u32 per lane; commands: 2 x u64 per lane (64 positions)
+    const uint4 e4 = ld_sys_v4(c.comp_ring + ((base + 4u * lane) & c.comp_mask));
+    const uint4 c4 = ld_sys_v4((const u32 *)(c.fcmd + ((cbase + 2u * lane) & c.ring_mask)));
+    bool progressed = false;
+    {
+      const u32 e[4] = {e4.x, e4.y, e4.z, e4.w};
+      u32 end;
+      ring_window(c, e, base, seen, lane, end);
+      u32 val[4]; bool take[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const u32 i = base + 4u * lane + (u32)k;
+        take[k] = i >= seen && i < end;
+        val[k] = e[k] >> 8;
+      }
+      bulk_push4(c, c.arr, val, take, end - seen, base + 4u * lane - seen, lane);
+      progressed |= end != seen;
+      seen = end;
+    }
+    {
+      const u64 w[2] = {((u64)c4.y << 32) | c4.x, ((u64)c4.w << 32) | c4.z};
+      u32 first_bad = 64;
+#pragma unroll
+      for (int k = 1; k >= 0; --k) {
+        const u32 i = cbase + 2u * lane + (u32)k;
+        const bool ok = ((u32)w[k] & 0xFFu) == ((i >> c.ring_shift) % 255u) + 1u || i < seen_cmd;
+        if (!ok) first_bad = 2u * lane + (u32)k;
+      }
+      const u32 end = cbase + __reduce_min_sync(0xffffffffu, first_bad);
+      u32 val[4] = {0, 0, 0, 0}; bool take[4] = {false, false, false, false};
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        const u32 i = cbase + 2u * lane + (u32)k;
+        take[k] = i >= seen_cmd && i < end;
+        val[k] = i;
+        if (take[k]) st_u64(c.fcmd_dev + (i & c.ring_mask), w[k]);
+      }
+      bulk_push4(c, c.cpy, val, take, end - seen_cmd, cbase + 2u * lane - seen_cmd, lane);
+      progressed |= end != seen_cmd;
+      seen_cmd = end;
+    }
+    if (!progressed) __nanosleep(100);
+    if ((++it & 15u) == 0) {
+      u32 abort_req = 0, late = 0;
+      if (lane == 0) {
+        abort_req = ld_sys_u32(c.host_ctl + 1);
+        late = globaltimer() - t0 > c.timeout_ns ? 1u : 0u;
+      }
+      if (__shfl_sync(0xffffffffu, abort_req, 0)) { if (lane == 0) raise(c, 5, 0xB1); break; }
+      if (__shfl_sync(0xffffffffu, late, 0)) { if (lane == 0) raise(c, 5, 0xB2); break; }
+    }
   }
 }
 
@@ -867,14 +1021,26 @@ __global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
   extern __shared__ u32 smem_lut[];
   const u32 lane = lane_id(), warp = threadIdx.x >> 5;
   if (blockIdx.x == 0 && warp == 0) { poller(c, lane); return; }
+  if (warp == (blockDim.x >> 5) - 1) { copier(c, lane); return; }
   u32 *lut = PQ ? smem_lut + (u64)warp * c.pq_m * kPqKsub : nullptr;
   const u64 t0 = globaltimer();
   u32 idle = 0;
+  // where the worker warps' time goes (ns, summed over warps): arrivals, query phases, idle
+  u64 t_arr = 0, t_run = 0, t_idle = 0, n_arr = 0, n_run = 0;
+  u64 tp = t0;
   for (;;) {
     if (warp_stopped(c)) break;
     u32 v;
-    if (warp_pop(c, c.arr, v, lane)) { consume_arrival(c, v, lane); idle = 0; continue; }
-    if (warp_pop(c, c.run, v, lane)) { run_query<PQ>(c, v, lane, lut); idle = 0; continue; }
+    if (warp_pop(c, c.arr, v, lane)) {
+      consume_arrival(c, v, lane); idle = 0;
+      const u64 t = globaltimer(); t_arr += t - tp; tp = t; ++n_arr;
+      continue;
+    }
+    if (warp_pop(c, c.run, v, lane)) {
+      run_query<PQ>(c, v, lane, lut); idle = 0;
+      const u64 t = globaltimer(); t_run += t - tp; tp = t; ++n_run;
+      continue;
+    }
     // nothing to run: see whether a page waiting for a slot can be given one
     if (lane == 0 && (int)ld_u32((const u32 *)c.want.count) > 0) {
       LaneStats st = {0, 0, 0, 0, 0, 0};
@@ -885,6 +1051,13 @@ __global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
     __nanosleep(idle < 16 ? 100 : 1000);
     u32 late = ((idle & 127u) == 0 && globaltimer() - t0 > c.timeout_ns) ? 1u : 0u;
     if (__shfl_sync(0xffffffffu, late, 0)) { if (lane == 0) raise(c, 5, 0xB3); break; }
+    { const u64 t = globaltimer(); t_idle += t - tp; tp = t; }
+  }
+  if (lane == 0) {
+    atomicAdd((unsigned long long *)&c.ctl->stats[S_T_ARR], t_arr);
+    atomicAdd((unsigned long long *)&c.ctl->stats[S_T_RUN], t_run);
+    atomicAdd((unsigned long long *)&c.ctl->stats[S_T_IDLE], t_idle);
+    atomicAdd((unsigned long long *)&c.ctl->stats[S_N_ARR], n_arr);
   }
 }
 
@@ -895,14 +1068,15 @@ __global__ void init_kernel(const Ctx c) {
   const u32 tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
   for (u32 i = tid; i < c.n_qslots; i += nth) reset_hdr(c.hdr + i, i);
   // runnable queue starts with every slot; the others start empty
-  u64 *run = (u64 *)c.run.buf, *arr = (u64 *)c.arr.buf, *want = (u64 *)c.want.buf;
+  u64 *run = (u64 *)c.run.buf, *arr = (u64 *)c.arr.buf, *want = (u64 *)c.want.buf, *cpy = (u64 *)c.cpy.buf;
+  for (u32 i = tid; i <= c.cpy.mask; i += nth) cpy[i] = (u64)i << 32;
   for (u32 i = tid; i <= c.run.mask; i += nth) run[i] = i < c.n_qslots ? (((u64)(i + 1u) << 32) | i) : ((u64)i << 32);
   for (u32 i = tid; i <= c.arr.mask; i += nth) arr[i] = (u64)i << 32;
   for (u32 i = tid; i <= c.want.mask; i += nth) want[i] = (u64)i << 32;
   if (tid == 0) {
     Ctl *ctl = c.ctl;
     ctl->stop = 0; ctl->status = 0; ctl->next_query = c.n_qslots; ctl->done = 0; ctl->ring_head = 0;
-    for (int i = 0; i < 12; ++i) ctl->q_heads[i] = 0;
+    for (int i = 0; i < 16; ++i) ctl->q_heads[i] = 0;
     for (int i = 0; i < 8; ++i) ctl->dbg[i] = 0;
     *c.run.tail = c.n_qslots;
     *c.run.count = (int)c.n_qslots;
@@ -921,42 +1095,19 @@ __global__ void cache_reset_kernel(const Ctx c, u32 preloaded) {
   if (tid == 0) { c.cs->bump = preloaded; c.cs->hand = 0; }
 }
 
-// Proxy copy batch: block b copies page b of the batch from host-mapped memory into its
-// cache slot (256 threads x 16 bytes); the last block to finish reports the batch sequence
-// number to the host.
-__global__ void fill_kernel(const FillBatch b, const u8 *host_pages, u8 *slot_data, u32 *counter,
-                            u32 *host_copied) {
-  const u32 i = blockIdx.x;
-  const uint4 *src = (const uint4 *)(host_pages + (u64)b.page[i] * kPageBytes);
-  uint4 *dst = (uint4 *)(slot_data + (u64)b.slot[i] * kPageBytes);
-  const uint4 v = __ldcs(src + threadIdx.x);
-  __stcg(dst + threadIdx.x, v);
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    u32 done = atomicAdd(counter, 1u) + 1u;
-    if (done == b.n) {
-      *counter = 0;
-      __threadfence_system();
-      asm volatile("st.relaxed.sys.global.u32 [%0], %1;" ::"l"(host_copied), "r"(b.seq) : "memory");
-    }
-  }
-}
-
 // ------------------------------------------------------------------------------------------
 // launchers
 // ------------------------------------------------------------------------------------------
 // With lazy module loading the first launch of a kernel may need a context-wide
-// synchronisation, which can never finish while the persistent kernel is waiting for that
-// very launch (the proxy's first copy kernel).  Querying the attributes loads the code now.
+// synchronisation; querying the attributes loads all code at open time instead, so that no
+// launch ever has to wait behind a resident persistent kernel.
 cudaError_t preload_kernels() {
   cudaFuncAttributes a;
   cudaError_t e;
   if ((e = cudaFuncGetAttributes(&a, search_kernel<false>)) != cudaSuccess) return e;
   if ((e = cudaFuncGetAttributes(&a, search_kernel<true>)) != cudaSuccess) return e;
   if ((e = cudaFuncGetAttributes(&a, init_kernel)) != cudaSuccess) return e;
-  if ((e = cudaFuncGetAttributes(&a, cache_reset_kernel)) != cudaSuccess) return e;
-  return cudaFuncGetAttributes(&a, fill_kernel);
+  return cudaFuncGetAttributes(&a, cache_reset_kernel);
 }
 
 cudaError_t launch_init(const Ctx &c, cudaStream_t s) {
@@ -990,12 +1141,6 @@ cudaError_t launch_search(const Ctx &c, u32 blocks, u32 warps_per_block, cudaStr
   } else {
     search_kernel<false><<<blocks, warps_per_block * 32, 0, s>>>(c);
   }
-  return cudaGetLastError();
-}
-
-cudaError_t launch_fill(const FillBatch &b, const u8 *host_pages_dev, u8 *slot_data, u32 *counter,
-                        u32 *host_copied, cudaStream_t s) {
-  fill_kernel<<<b.n, 256, 0, s>>>(b, host_pages_dev, slot_data, counter, host_copied);
   return cudaGetLastError();
 }
 

@@ -102,13 +102,13 @@ def test_cold_cache_with_room_for_every_page_fetches_each_page_once(gorio, cfg1)
 @pytest.mark.parametrize("cfg", [
     dict(capacity=16), dict(capacity=64, max_outstanding=1), dict(capacity=1000, remote_latency_ns=20000),
     dict(capacity=1000, remote_latency_ns=200000, max_outstanding=32),
-    dict(capacity=1000, fill_batch=1), dict(capacity=1000, fill_batch=128, max_outstanding=1024),
+    dict(capacity=1000, max_outstanding=4), dict(capacity=1000, max_outstanding=1024),
     dict(capacity=2500, tuning=dict(warps_per_block=4)), dict(capacity=2500, tuning=dict(max_inflight=48)),
     dict(capacity=2500, tuning=dict(warps_per_block=8, blocks_per_sm=2)),
 ], ids=lambda c: "-".join(f"{k}={v}" for k, v in c.items() if k != "tuning") + ("-tuned" if "tuning" in c else ""))
 def test_results_do_not_depend_on_cache_proxy_or_geometry(gorio, cfg1, cfg):
     """The proxy never touches search state, so outputs must be identical under any cache
-    size, latency, outstanding depth, batch size and launch geometry."""
+    size, latency, outstanding depth and launch geometry."""
     w, ref = cfg1
     cfg = dict(cfg)
     cap = cfg.pop("capacity")
