@@ -137,9 +137,9 @@ typedef struct {
   uint64_t proxy_service_ns, proxy_iters, proxy_ack_wait_iters, proxy_window_full_iters;
   uint64_t proxy_ring_empty_iters, proxy_outstanding_sum;
   /* where the worker warps' time went, ns summed over warps: serving arrived pages,
-     running query phases, idle; and the number of arrival-queue items consumed */
+     running query phases, idle; the number of arrival-queue items consumed; ns executing copy commands */
   uint64_t warp_ns_arrivals, warp_ns_queries, warp_ns_idle, arrivals_consumed;
-  uint64_t reserved1, reserved2;
+  uint64_t warp_ns_copies, reserved2;
 } gorio_stats_t;
 
 /* Open an index on CUDA device `cuda_device`.  *out is set only on GORIO_OK. */

@@ -51,7 +51,7 @@ _STAT_FIELDS = ["pages_hit", "pages_missed", "pages_fetched", "dedupe_joins", "e
                 "resumes", "search_ns", "proxy_batches", "posted", "proxy_service_ns", "proxy_iters",
                 "proxy_ack_wait_iters", "proxy_window_full_iters", "proxy_ring_empty_iters",
                 "proxy_outstanding_sum", "warp_ns_arrivals", "warp_ns_queries", "warp_ns_idle",
-                "arrivals_consumed", "reserved1", "reserved2"]
+                "arrivals_consumed", "warp_ns_copies", "reserved2"]
 
 
 class Stats(ctypes.Structure):
@@ -99,7 +99,8 @@ class Index:
 
     def __init__(self, pages: np.ndarray, n_nodes: int, dim: int, dtype: str, max_degree: int,
                  nodes_per_page: int, entry_id: int, device: int = 0,
-                 pq_centroids: Optional[torch.Tensor] = None, pq_codes: Optional[torch.Tensor] = None):
+                 pq_centroids: Optional[torch.Tensor] = None, pq_codes: Optional[torch.Tensor] = None,
+                 already_pinned: bool = False):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         assert pages.dtype == np.uint8 and pages.flags["C_CONTIGUOUS"]
@@ -111,6 +112,7 @@ class Index:
         d.n_nodes, d.dim, d.dtype = n_nodes, dim, 0 if self.dtype == "u8" else 1
         d.max_degree, d.nodes_per_page, d.page_bytes, d.entry_id = max_degree, nodes_per_page, 4096, entry_id
         d.host_pages = pages.ctypes.data
+        d.flags = 1 if already_pinned else 0
         if pq_centroids is not None:
             assert pq_centroids.is_cuda and pq_codes.is_cuda and pq_centroids.dtype == torch.uint8
             d.pq_m = pq_centroids.shape[0]
@@ -118,12 +120,20 @@ class Index:
         self._check(self._lib.gorio_index_open(ctypes.byref(d), device, ctypes.byref(self._h)), opened=False)
 
     @classmethod
-    def from_workload(cls, w, device=0, use_pq=False):
+    def from_workload(cls, w, device=0, use_pq=False, pin=False):
+        """pin=True copies the page store into CUDA-allocated pinned memory first (instead of
+        page-locking the numpy buffer in place)."""
         cent = codes = None
         if use_pq:
             cent = torch.as_tensor(w.pq_centroids).contiguous().cuda(device)
             codes = torch.as_tensor(w.pq_codes).contiguous().cuda(device)
-        return cls(w.pages, w.N, w.d, w.dtype, w.R, w.npp, w.entry, device, cent, codes)
+        pages, keep = w.pages, None
+        if pin:
+            keep = torch.from_numpy(w.pages).pin_memory()
+            pages = keep.numpy()
+        ix = cls(pages, w.N, w.d, w.dtype, w.R, w.npp, w.entry, device, cent, codes, already_pinned=pin)
+        ix._pinned_store = keep
+        return ix
 
     def _check(self, status, opened=True):
         if status != 0:

@@ -45,7 +45,7 @@ struct gorio_index {
   u32 n_slots = 0, preloaded = 0;
   u8 *slot_data = nullptr;
   u64 *ptab = nullptr, *smeta = nullptr;
-  u32 *parts = nullptr;
+  u32 *parts = nullptr, *filled = nullptr;
   CacheShared *cs = nullptr;
   u64 *want_buf = nullptr; u32 want_cap = 0;
   u64 *cpy_buf = nullptr, *fcmd_mirror = nullptr;
@@ -117,7 +117,7 @@ cudaError_t host_mapped(T **h, T **d, size_t count) {
 }
 
 void free_cache(gorio_index *ix) {
-  cudaFree(ix->slot_data); cudaFree(ix->ptab); cudaFree(ix->smeta); cudaFree(ix->parts); cudaFree(ix->cs);
+  cudaFree(ix->slot_data); cudaFree(ix->ptab); cudaFree(ix->smeta); cudaFree(ix->parts); cudaFree(ix->filled); cudaFree(ix->cs);
   cudaFree(ix->want_buf); cudaFree(ix->cpy_buf); cudaFree(ix->fcmd_mirror);
   ix->cpy_buf = ix->fcmd_mirror = nullptr;
   if (ix->ring_h) cudaFreeHost(ix->ring_h);
@@ -125,7 +125,7 @@ void free_cache(gorio_index *ix) {
   if (ix->fcmd_h) cudaFreeHost(ix->fcmd_h);
   if (ix->fdone_h) cudaFreeHost(ix->fdone_h);
   ix->fcmd_h = ix->fcmd_d = nullptr; ix->fdone_h = ix->fdone_d = nullptr;
-  ix->slot_data = nullptr; ix->ptab = ix->smeta = nullptr; ix->parts = nullptr; ix->cs = nullptr;
+  ix->slot_data = nullptr; ix->ptab = ix->smeta = nullptr; ix->parts = ix->filled = nullptr; ix->cs = nullptr;
   ix->want_buf = nullptr;
   ix->ring_h = ix->ring_d = nullptr; ix->comp_h = ix->comp_d = nullptr;
   ix->cache_ready = false;
@@ -264,6 +264,7 @@ int setup_cache(gorio_index *ix) {
   CK(cudaMalloc(&ix->ptab, (size_t)ix->n_pages * 8));
   CK(cudaMalloc(&ix->smeta, (size_t)ix->n_slots * 8));
   CK(cudaMalloc(&ix->parts, (size_t)ix->n_slots * 4));
+  CK(cudaMalloc(&ix->filled, (size_t)ix->n_slots * 4));
   CK(cudaMalloc(&ix->cs, sizeof(CacheShared)));
   CK(cudaMalloc(&ix->want_buf, (size_t)ix->want_cap * 8));
   CK(cudaMalloc(&ix->cpy_buf, (size_t)ix->ring_cap * 8));
@@ -278,7 +279,7 @@ int setup_cache(gorio_index *ix) {
     CK(cudaMemcpy(ix->slot_data, ix->desc.host_pages, (size_t)ix->preloaded * kPageBytes, cudaMemcpyHostToDevice));
   }
   Ctx c{};
-  c.ptab = ix->ptab; c.smeta = ix->smeta; c.parts = ix->parts; c.cs = ix->cs;
+  c.ptab = ix->ptab; c.smeta = ix->smeta; c.parts = ix->parts; c.filled = ix->filled; c.cs = ix->cs;
   c.n_slots = ix->n_slots; c.n_pages = ix->n_pages;
   CK(launch_cache_reset(c, ix->preloaded, ix->own_stream));
   CK(cudaStreamSynchronize(ix->own_stream));
@@ -468,7 +469,7 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   c.n_nodes = (u32)d.n_nodes; c.dim = d.dim; c.dtype = d.dtype; c.R = d.max_degree; c.npp = d.nodes_per_page;
   c.node_bytes = ix->node_bytes; c.vec_bytes = ix->vec_bytes; c.entry = d.entry_id; c.n_pages = ix->n_pages;
   c.pq_m = d.pq_m; c.pq_dsub = d.pq_m ? d.dim / d.pq_m : 0; c.pq_cent = d.pq_centroids_dev; c.pq_codes = d.pq_codes_dev;
-  c.slot_data = ix->slot_data; c.ptab = ix->ptab; c.smeta = ix->smeta; c.parts = ix->parts; c.cs = ix->cs;
+  c.slot_data = ix->slot_data; c.ptab = ix->ptab; c.smeta = ix->smeta; c.parts = ix->parts; c.filled = ix->filled; c.cs = ix->cs;
   c.n_slots = ix->n_slots;
   c.ring = ix->ring_d; c.ring_mask = ix->ring_cap - 1; c.ring_shift = ilog2(ix->ring_cap);
   c.comp_ring = ix->comp_d; c.comp_mask = ix->ring_cap - 1; c.host_ctl = ix->hctl_d;
@@ -489,10 +490,9 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
 
   // launch geometry: leave room on every SM for the proxy's copy kernels
   const bool pq = d.pq_m != 0;
-  // warps per block = worker warps + one copier warp (block 0 also hosts the completion poller)
-  u32 warps = (ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 5u : 16u)) + 1u;
+  u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 6u : 16u);
   if (pq) { u32 lim = (200u * 1024u) / (d.pq_m * kPqKsub * 4u); if (warps > lim) warps = lim; }
-  if (warps < 3) return fail(ix, GORIO_ERR_INVALID_ARG, "search: shared memory cannot hold the PQ tables of a block");
+  if (warps < 3) return fail(ix, GORIO_ERR_INVALID_ARG, "search: need at least 3 warps per block (two pollers and a worker)");
   int occ = 0;
   CK(search_occupancy(d.pq_m, warps, &occ));
   if (occ < 1) return fail(ix, GORIO_ERR_INVALID_ARG, "search: launch geometry does not fit an SM");
@@ -595,7 +595,7 @@ int gorio_stats(gorio_index *ix, gorio_stats_t *out) {
   out->proxy_window_full_iters = ix->host_window_full; out->proxy_ring_empty_iters = ix->host_ring_empty;
   out->proxy_iters = ix->host_iters; out->proxy_outstanding_sum = ix->host_out_sum;
   out->warp_ns_arrivals = h.stats[S_T_ARR]; out->warp_ns_queries = h.stats[S_T_RUN]; out->warp_ns_idle = h.stats[S_T_IDLE];
-  out->arrivals_consumed = h.stats[S_N_ARR];
+  out->arrivals_consumed = h.stats[S_N_ARR]; out->warp_ns_copies = h.stats[S_T_CPY];
   return GORIO_OK;
 }
 

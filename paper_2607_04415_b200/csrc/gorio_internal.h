@@ -60,11 +60,11 @@ struct Ctl {
   u32 q_heads[16]; // queue head/tail/count words: arr(0,1,2) run(3,4,5) want(6,7,8) copy(9,10,11)
   u32 dbg[8];      // detail of the first error
   u32 census[16];  // debug snapshot (see census())
-  u64 stats[16];
+  u64 stats[32];
 };
 
 enum StatIdx { S_HIT = 0, S_MISSED, S_JOINS, S_EVICT, S_RETRY, S_DONE, S_NEVAL, S_NEXPAND,
-               S_SUMDEG, S_NITER, S_RESUMES, S_POSTED, S_T_ARR, S_T_RUN, S_T_IDLE, S_N_ARR };
+               S_SUMDEG, S_NITER, S_RESUMES, S_POSTED, S_T_ARR, S_T_RUN, S_T_IDLE, S_N_ARR, S_T_CPY };
 
 // Everything the persistent kernel needs, passed by value.
 struct Ctx {
@@ -78,6 +78,7 @@ struct Ctx {
   u64 *ptab;       // [n_pages] page words: state, slot, waiter-list head or generation
   u64 *smeta;      // [n_slots] slot words: page, generation, reference bit
   u32 *parts;      // [n_slots] waiter-chain segments still being served
+  u32 *filled;     // [n_slots] generation whose bytes the copier has stored into the slot
   CacheShared *cs; // clock hand and bump pointer
   u32 n_slots;
   // miss ring: host-mapped, written by the GPU, consumed by the proxy

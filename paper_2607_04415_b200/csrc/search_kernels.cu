@@ -388,6 +388,17 @@ __device__ void consume_arrival(const Ctx &c, u32 v, u32 lane) {
   if (page >= c.n_pages) { if (lane == 0) raise(c, 8, 0x76, slot, page); return; }
   u32 head = 0, bad = 0;
   if (lane == 0) {
+    // acquire the copier's stores into the slot (normally long done: the completion was
+    // published at least the remote latency after the bytes arrived)
+    u32 spins = 0;
+    while (ld_u32(c.filled + slot) != gen) {
+      __nanosleep(100);
+      if (++spins > (1u << 20)) { raise(c, 5, 0x77, slot, gen); bad = 1; break; }
+    }
+    __threadfence();
+  }
+  if (__shfl_sync(0xffffffffu, bad, 0)) return;
+  if (lane == 0) {
     st_u32(c.parts + slot, 1u);
     st_u64(c.smeta + slot, m | 1ull);                      // a fresh page gets its second chance
     __threadfence();
@@ -845,56 +856,50 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut) {
   if (lane == 0) raise(c, 6, 0xA2, qs);
 }
 
-// Copier warps (the last warp of every block) execute the proxy's copy commands, which the
-// poller mirrors into device memory: pull the 4 KB page from the pinned store into the cache
-// slot (each lane moves 8 x 16 bytes, all loads in flight before the first store) and
-// acknowledge to the host, which publishes the completion once the latency has elapsed.
-// Only the page bytes cross the host link on this path; no copier ever polls host memory.
-__device__ void copier(const Ctx &c, u32 lane) {
-  u32 idle = 0;
-  const u64 t0 = globaltimer();
-  for (;;) {
-    if (warp_stopped(c)) break;
-    u32 idx;
-    if (!warp_pop(c, c.cpy, idx, lane)) {
-      ++idle;
-      __nanosleep(idle < 64 ? 100 : 1000);
-      u32 late = ((idle & 255u) == 0 && globaltimer() - t0 > c.timeout_ns) ? 1u : 0u;
-      if (__shfl_sync(0xffffffffu, late, 0)) { if (lane == 0) raise(c, 5, 0xB4); break; }
-      continue;
-    }
-    idle = 0;
-    const u64 cmd = __shfl_sync(0xffffffffu, ld_u64(c.fcmd_dev + (idx & c.ring_mask)), 0);
-    const u32 page = (u32)(cmd >> 32), slot = (u32)(cmd >> 8) & 0xFFFFFFu;
-    if (page >= c.n_pages || slot >= c.n_slots) { if (lane == 0) raise(c, 8, 0xC1, idx, page, slot); break; }
-    const uint4 *src = (const uint4 *)(c.host_pages + (u64)page * kPageBytes);
-    uint4 *dst = (uint4 *)(c.slot_data + (u64)slot * kPageBytes);
-    uint4 v[8];
+// Execute one of the proxy's copy commands (mirrored into device memory by the poller): pull
+// the 4 KB page from the pinned store into its cache slot.  Any worker warp does this, ahead
+// of all other work; only the page bytes cross the host link on this path.  The host is told
+// as soon as the page's bytes have arrived on the GPU (they are in registers), so that no
+// fence sits inside the proxy's outstanding window; the stores into the slot are then
+// released to the consumers of the arrival through the slot's `filled` generation.
+__device__ void copy_page(const Ctx &c, u32 idx, u32 lane) {
+  const u64 cmd = __shfl_sync(0xffffffffu, ld_u64(c.fcmd_dev + (idx & c.ring_mask)), 0);
+  const u32 page = (u32)(cmd >> 32), slot = (u32)(cmd >> 8) & 0xFFFFFFu;
+  if (page >= c.n_pages || slot >= c.n_slots) { if (lane == 0) raise(c, 8, 0xC1, idx, page, slot); return; }
+  const uint4 *src = (const uint4 *)(c.host_pages + (u64)page * kPageBytes);
+  uint4 *dst = (uint4 *)(c.slot_data + (u64)slot * kPageBytes);
+  uint4 v[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = __ldcs(src + i * 32 + lane);
+  for (int i = 0; i < 8; ++i) v[i] = __ldcs(src + i * 32 + lane);
+  // a value that depends on every loaded word: the acknowledgement cannot be issued early
+  u32 dep = 0;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) __stcg(dst + i * 32 + lane, v[i]);
+  for (int i = 0; i < 8; ++i) dep |= (v[i].x ^ v[i].x);
+  dep = __reduce_or_sync(0xffffffffu, dep);
+  if (lane == 0) st_sys_u32(c.fdone + (idx & c.ring_mask), ((u32)cmd & 0xFFu) | dep);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) __stcg(dst + i * 32 + lane, v[i]);
+  __syncwarp();          // orders every lane's stores before lane 0's release below
+  if (lane == 0) {
+    const u32 gen = sm_gen(ld_u64(c.smeta + slot));
     __threadfence();
-    __syncwarp();
-    if (lane == 0) {
-      __threadfence_system();
-      st_sys_u32(c.fdone + (idx & c.ring_mask), (u32)cmd & 0xFFu);
-    }
+    st_u32(c.filled + slot, gen);
   }
 }
 
-// Push n values (lane-distributed: value k of this lane goes to position rank0 + k if
-// take[k]) with one ticket reservation and one count update for the whole warp.
-__device__ __forceinline__ void bulk_push4(const Ctx &c, const Queue &q, const u32 (&val)[4], const bool (&take)[4],
-                                           u32 n, u32 first_rank, u32 lane) {
+// Push n values with one ticket reservation and one count update for the whole warp: value k
+// of this lane goes to position ofs[k] (0 <= ofs < n, all distinct) if take[k].
+template <int NV>
+__device__ __forceinline__ void bulk_push(const Ctx &c, const Queue &q, const u32 (&val)[NV], const u32 (&ofs)[NV],
+                                          const bool (&take)[NV], u32 n, u32 lane) {
   if (n == 0) return;
   u32 base = 0;
   if (lane == 0) { __threadfence(); base = atomicAdd(q.tail, n); }
   base = __shfl_sync(0xffffffffu, base, 0);
 #pragma unroll
-  for (int k = 0; k < 4; ++k) {
+  for (int k = 0; k < NV; ++k) {
     if (take[k]) {
-      const u32 pos = base + first_rank + (u32)k;
+      const u32 pos = base + ofs[k];
       u64 *cell = (u64 *)q.buf + (pos & q.mask);
       u32 spins = 0;
       while ((u32)(ld_u64(cell) >> 32) != pos) {
@@ -905,22 +910,6 @@ __device__ __forceinline__ void bulk_push4(const Ctx &c, const Queue &q, const u
   }
   __syncwarp();
   if (lane == 0) atomicAdd(q.count, (int)n);
-}
-
-// Warp 0 of block 0 is the only warp that reads control data from host memory.  Per
-// iteration it reads the next 128 positions of the proxy's completion ring and of its
-// copy-command ring (both self-validating through a lap tag, one 512-byte read each, issued
-// together), forwards new completions to the arrival queue and new commands, mirrored
-// into device memory, to the copy queue.  The abort word is sampled now and then.
-__device__ void ring_window(const Ctx &c, const u32 (&e)[4], u32 base, u32 seen, u32 lane, u32 &end) {
-  u32 first_bad = 128;
-#pragma unroll
-  for (int k = 3; k >= 0; --k) {
-    const u32 i = base + 4u * lane + (u32)k;
-    const bool ok = (e[k] & 0xFFu) == ((i >> c.ring_shift) % 255u) + 1u || i < seen;
-    if (!ok) first_bad = 4u * lane + (u32)k;
-  }
-  end = base + __reduce_min_sync(0xffffffffu, first_bad);    // entries [seen, end) are new and valid
 }
 
 // Debug aid: one snapshot of where slots, pages and queries are, taken by the poller warp.
@@ -952,56 +941,65 @@ __device__ void census(const Ctx &c, u32 lane) {
   }
 }
 
-__device__ void poller(const Ctx &c, u32 lane) {
-  u32 seen = 0, seen_cmd = 0, it = 0;
+// Two poller warps are the only warps that read control data from host memory: warp 0 of
+// block 0 follows the proxy's completion ring, warp 0 of block 1 (or warp 1 of block 0 in a
+// one-block launch) its copy-command ring.  Ring entries are self-validating through a lap
+// tag, so per iteration a poller reads the next 256 ring positions with fully coalesced
+// 512-byte warp loads and forwards the valid prefix in bulk: completions to the arrival
+// queue; commands, mirrored into device memory, to the copy queue.  The abort word is
+// sampled now and then.
+constexpr u32 kPollWidth = 256;
+
+__device__ void poller(const Ctx &c, bool commands, u32 lane) {
+  u32 seen = 0, it = 0;
   const u64 t0 = globaltimer();
-  bool census_done = c.census_ns == 0;
+  bool census_done = c.census_ns == 0 || commands;
   for (;;) {
     if (warp_stopped(c)) break;
     if (!census_done && globaltimer() - t0 > c.census_ns) { census(c, lane); census_done = true; }
-    const u32 base = seen & ~3u, cbase = seen_cmd & ~1u;
-    // completions: 4 x u32 per lane; commands: 2 x u64 per lane (64 positions)
-    const uint4 e4 = ld_sys_v4(c.comp_ring + ((base + 4u * lane) & c.comp_mask));
-    const uint4 c4 = ld_sys_v4((const u32 *)(c.fcmd + ((cbase + 2u * lane) & c.ring_mask)));
-    bool progressed = false;
-    {
-      const u32 e[4] = {e4.x, e4.y, e4.z, e4.w};
-      u32 end;
-      ring_window(c, e, base, seen, lane, end);
-      u32 val[4]; bool take[4];
+    const u32 base = seen & ~7u;        // 8 | base keeps every 16-byte load inside the ring
+    u32 val[8], rel[8]; bool take[8]; u32 first_bad = kPollWidth;
+    u64 w[8];
+    if (!commands) {
+      // load k covers ring positions base + 128k + [0,128): lane l gets 4 of them
+      uint4 q4[2];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const u32 i = base + 4u * lane + (u32)k;
-        take[k] = i >= seen && i < end;
-        val[k] = e[k] >> 8;
-      }
-      bulk_push4(c, c.arr, val, take, end - seen, base + 4u * lane - seen, lane);
-      progressed |= end != seen;
-      seen = end;
-    }
-    {
-      const u64 w[2] = {((u64)c4.y << 32) | c4.x, ((u64)c4.w << 32) | c4.z};
-      u32 first_bad = 64;
-#pragma unroll
-      for (int k = 1; k >= 0; --k) {
-        const u32 i = cbase + 2u * lane + (u32)k;
-        const bool ok = ((u32)w[k] & 0xFFu) == ((i >> c.ring_shift) % 255u) + 1u || i < seen_cmd;
-        if (!ok) first_bad = 2u * lane + (u32)k;
-      }
-      const u32 end = cbase + __reduce_min_sync(0xffffffffu, first_bad);
-      u32 val[4] = {0, 0, 0, 0}; bool take[4] = {false, false, false, false};
+      for (int k = 0; k < 2; ++k) q4[k] = ld_sys_v4(c.comp_ring + ((base + 128u * k + 4u * lane) & c.comp_mask));
 #pragma unroll
       for (int k = 0; k < 2; ++k) {
-        const u32 i = cbase + 2u * lane + (u32)k;
-        take[k] = i >= seen_cmd && i < end;
-        val[k] = i;
-        if (take[k]) st_u64(c.fcmd_dev + (i & c.ring_mask), w[k]);
+        const u32 e[4] = {q4[k].x, q4[k].y, q4[k].z, q4[k].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { rel[4 * k + j] = 128u * k + 4u * lane + j; val[4 * k + j] = e[j] >> 8; w[4 * k + j] = e[j]; }
       }
-      bulk_push4(c, c.cpy, val, take, end - seen_cmd, cbase + 2u * lane - seen_cmd, lane);
-      progressed |= end != seen_cmd;
-      seen_cmd = end;
+    } else {
+      // load k covers ring positions base + 64k + [0,64): lane l gets 2 of them
+      uint4 q4[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) q4[k] = ld_sys_v4((const u32 *)(c.fcmd + ((base + 64u * k + 2u * lane) & c.ring_mask)));
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        w[2 * k] = ((u64)q4[k].y << 32) | q4[k].x; w[2 * k + 1] = ((u64)q4[k].w << 32) | q4[k].z;
+        rel[2 * k] = 64u * k + 2u * lane; rel[2 * k + 1] = rel[2 * k] + 1u;
+      }
     }
-    if (!progressed) __nanosleep(100);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const u32 i = base + rel[k];
+      const bool ok = ((u32)w[k] & 0xFFu) == ((i >> c.ring_shift) % 255u) + 1u || i < seen;
+      if (!ok && rel[k] < first_bad) first_bad = rel[k];
+    }
+    const u32 end = base + __reduce_min_sync(0xffffffffu, first_bad);   // [seen, end) new and valid
+    u32 ofs[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const u32 i = base + rel[k];
+      take[k] = i >= seen && i < end;
+      ofs[k] = i - seen;
+      if (commands) { val[k] = i; if (take[k]) st_u64(c.fcmd_dev + (i & c.ring_mask), w[k]); }
+    }
+    bulk_push<8>(c, commands ? c.cpy : c.arr, val, ofs, take, end - seen, lane);
+    if (end == seen) __nanosleep(100);
+    seen = end;
     if ((++it & 15u) == 0) {
       u32 abort_req = 0, late = 0;
       if (lane == 0) {
@@ -1020,17 +1018,22 @@ template <bool PQ>
 __global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
   extern __shared__ u32 smem_lut[];
   const u32 lane = lane_id(), warp = threadIdx.x >> 5;
-  if (blockIdx.x == 0 && warp == 0) { poller(c, lane); return; }
-  if (warp == (blockDim.x >> 5) - 1) { copier(c, lane); return; }
+  if (blockIdx.x == 0 && warp == 0) { poller(c, false, lane); return; }
+  if ((gridDim.x > 1 && blockIdx.x == 1 && warp == 0) || (gridDim.x == 1 && warp == 1)) { poller(c, true, lane); return; }
   u32 *lut = PQ ? smem_lut + (u64)warp * c.pq_m * kPqKsub : nullptr;
   const u64 t0 = globaltimer();
   u32 idle = 0;
   // where the worker warps' time goes (ns, summed over warps): arrivals, query phases, idle
-  u64 t_arr = 0, t_run = 0, t_idle = 0, n_arr = 0, n_run = 0;
+  u64 t_arr = 0, t_run = 0, t_idle = 0, t_cpy = 0, n_arr = 0, n_run = 0;
   u64 tp = t0;
   for (;;) {
     if (warp_stopped(c)) break;
     u32 v;
+    if (warp_pop(c, c.cpy, v, lane)) {           // the outstanding window waits on these
+      copy_page(c, v, lane); idle = 0;
+      const u64 t = globaltimer(); t_cpy += t - tp; tp = t;
+      continue;
+    }
     if (warp_pop(c, c.arr, v, lane)) {
       consume_arrival(c, v, lane); idle = 0;
       const u64 t = globaltimer(); t_arr += t - tp; tp = t; ++n_arr;
@@ -1058,6 +1061,7 @@ __global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
     atomicAdd((unsigned long long *)&c.ctl->stats[S_T_RUN], t_run);
     atomicAdd((unsigned long long *)&c.ctl->stats[S_T_IDLE], t_idle);
     atomicAdd((unsigned long long *)&c.ctl->stats[S_N_ARR], n_arr);
+    atomicAdd((unsigned long long *)&c.ctl->stats[S_T_CPY], t_cpy);
   }
 }
 
@@ -1091,6 +1095,7 @@ __global__ void cache_reset_kernel(const Ctx c, u32 preloaded) {
   for (u32 s = tid; s < c.n_slots; s += nth) {
     c.smeta[s] = s < preloaded ? mk_sm(s, 1, 1) : mk_sm(kInvalidId, 0, 0);
     c.parts[s] = 0;
+    c.filled[s] = s < preloaded ? 1u : 0u;
   }
   if (tid == 0) { c.cs->bump = preloaded; c.cs->hand = 0; }
 }
