@@ -191,9 +191,48 @@ int gorio_stats_reset(gorio_index *ix);
 /* Stops the proxy thread, frees every device and host resource of the index. */
 int gorio_index_close(gorio_index *ix);
 
+/*
+ * Search for callers that cannot allocate (the paper has no counterpart: this is a
+ * packaging variant of gorio_search, not a step of its method).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- services whose device
+ * memory is a pre-sized arena with every byte accounted for, latency-critical loops that
+ * cannot take the allocator's implicit device synchronisation, plugins whose host forbids
+ * allocation after start-up.  gorio_index_open / gorio_cache_config / gorio_search allocate
+ * device and pinned memory; this call allocates nothing, on the device or on the host, and
+ * needs no index handle.
+ *
+ * What it does: the same beam search (exact navigation only, pq_m must be 0), by the same
+ * kernels, over an index whose pages are ALL resident in device memory, so there are no
+ * misses and no proxy.  All working state comes from one fixed 12 MiB device array that is
+ * part of the library image: every GPU context that loads the library carries it until the
+ * process exits.
+ *
+ *   desc        index description; host_pages, flags and the PQ pointers are ignored.
+ *   pages_dev   DEVICE, n_pages * 4096 bytes in the page-store format, 16-byte aligned, read only.
+ *   queries_dev, out_ids_dev, out_dists_dev, out_pages_distinct_dev (may be NULL), cuda_stream:
+ *               as for gorio_search.  Runs on the CURRENT device; all pointers must belong to it.
+ * Limits (fixed by the array's size; beyond them the call returns GORIO_ERR_INVALID_ARG and
+ * gorio_last_error(NULL) says which): at most 32768 pages (128 MiB of index),
+ * 1 <= K <= L <= 256, W <= 16, W * max_degree <= 256.  At most 64 queries are in flight at a
+ * time (any nq is accepted).  A query that visits more than 16384 nodes fails the call with
+ * GORIO_ERR_CAPACITY.
+ * Sharing: every call on a GPU uses the same array, which still holds the previous call's
+ * state; the call re-initialises what must start clean.  Calls whose kernels overlap on one
+ * GPU race on it -- serialise them.  The call blocks until its kernel has finished.
+ * First call on a device: it also resolves the array's device address
+ * (cudaGetSymbolAddress) and loads the kernels; make that first call before any stream
+ * capture begins.
+ */
+int gorio_search_resident_noalloc(const gorio_index_desc *desc, const void *pages_dev,
+                                  const void *queries_dev, uint32_t nq, uint32_t K, uint32_t L,
+                                  uint32_t W, uint32_t *out_ids_dev, void *out_dists_dev,
+                                  uint32_t *out_pages_distinct_dev, void *cuda_stream);
+
 /* Static strings; never NULL. */
 const char *gorio_status_str(int status);
-/* Human-readable detail of the last non-OK status on this index (valid until the next call). */
+/* Human-readable detail of the last non-OK status on this index (valid until the next call);
+ * with ix == NULL, of the last failed call of this thread that takes no index handle. */
 const char *gorio_last_error(gorio_index *ix);
 
 #ifdef __cplusplus

@@ -11,4 +11,5 @@ from .binding import (  # noqa: F401
     lib_path,
     load_library,
     EXPORTED_SYMBOLS,
+    search_resident_noalloc,
 )

@@ -14,6 +14,7 @@ _LIB = None
 EXPORTED_SYMBOLS = [
     "gorio_index_open", "gorio_cache_config", "gorio_set_tuning", "gorio_search", "gorio_search_host",
     "gorio_stats", "gorio_stats_reset", "gorio_index_close", "gorio_status_str", "gorio_last_error",
+    "gorio_search_resident_noalloc",
 ]
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "CUDA", 3: "NOMEM", 4: "STATE", 5: "TIMEOUT",
@@ -80,6 +81,7 @@ def load_library():
     lib.gorio_set_tuning.argtypes = [vp, ctypes.POINTER(_Tuning)]
     lib.gorio_search.argtypes = [vp, vp, u32, u32, u32, u32, vp, vp, vp, vp, vp]
     lib.gorio_search_host.argtypes = [vp, vp, u32, u32, u32, u32, vp, vp, vp, vp]
+    lib.gorio_search_resident_noalloc.argtypes = [ctypes.POINTER(_IndexDesc), vp, vp, u32, u32, u32, u32, vp, vp, vp, vp]
     lib.gorio_stats.argtypes = [vp, ctypes.POINTER(Stats)]
     lib.gorio_stats_reset.argtypes = [vp]
     lib.gorio_index_close.argtypes = [vp]
@@ -198,3 +200,30 @@ class Index:
             self.close()
         except Exception:
             pass
+
+
+def search_resident_noalloc(pages_dev: torch.Tensor, n_nodes: int, dim: int, dtype: str, max_degree: int,
+                            nodes_per_page: int, entry_id: int, queries: torch.Tensor, K: int, L: int, W: int,
+                            stream=None):
+    """gorio_search_resident_noalloc: search an index that is fully resident in device memory
+    without any allocation inside the library (the result tensors are allocated here, by the
+    caller's allocator, before the call).  For callers that cannot call cudaMalloc; limits
+    and sharing rules are in include/gorio.h."""
+    lib = load_library()
+    assert pages_dev.is_cuda and pages_dev.dtype == torch.uint8 and pages_dev.is_contiguous()
+    assert queries.is_cuda and queries.is_contiguous()
+    u8 = str(dtype) in ("u8", "uint8")
+    d = _IndexDesc()
+    d.n_nodes, d.dim, d.dtype = n_nodes, dim, 0 if u8 else 1
+    d.max_degree, d.nodes_per_page, d.page_bytes, d.entry_id = max_degree, nodes_per_page, 4096, entry_id
+    nq, dev = queries.shape[0], queries.device
+    ids = torch.empty((nq, K), dtype=torch.int32, device=dev)
+    dists = torch.empty((nq, K), dtype=torch.int32 if u8 else torch.float32, device=dev)
+    pages = torch.empty(nq, dtype=torch.int32, device=dev)
+    s = stream if stream is not None else torch.cuda.current_stream(dev)
+    with torch.cuda.device(dev):
+        st = lib.gorio_search_resident_noalloc(ctypes.byref(d), pages_dev.data_ptr(), queries.data_ptr(), nq, K, L, W,
+                                               ids.data_ptr(), dists.data_ptr(), pages.data_ptr(), s.cuda_stream)
+    if st != 0:
+        raise GorioError(st, lib.gorio_last_error(None).decode())
+    return dict(ids=ids, dists=dists, pages_distinct=pages)

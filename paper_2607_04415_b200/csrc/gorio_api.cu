@@ -329,10 +329,19 @@ int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W) {
   return GORIO_OK;
 }
 
+thread_local char g_global_error[256] = "";
+
 const char *kDeviceErr[] = {"", "", "", "", "", "device wait expired", "per-query capacity exhausted",
                             "corrupt index page", "internal state-machine check failed"};
 
 }  // namespace
+
+namespace gorio {
+// message of the last failed call that has no index handle (this thread)
+void set_global_error(const char *msg) {
+  std::snprintf(g_global_error, sizeof g_global_error, "%s", msg ? msg : "");
+}
+}  // namespace gorio
 
 // =========================================================================================
 extern "C" {
@@ -352,7 +361,7 @@ const char *gorio_status_str(int s) {
   }
 }
 
-const char *gorio_last_error(gorio_index *ix) { return ix ? ix->err.c_str() : ""; }
+const char *gorio_last_error(gorio_index *ix) { return ix ? ix->err.c_str() : g_global_error; }
 
 int gorio_index_open(const gorio_index_desc *d, int cuda_device, gorio_index **out) {
   if (!d || !out) return GORIO_ERR_INVALID_ARG;
