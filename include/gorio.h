@@ -104,13 +104,19 @@ typedef struct {
  *   max_inflight     query slots resident at once (pending/running queries); default 16384.
  *   visited_capacity per-query exact visited-set entries (power of two), default 32768;
  *                    a query that scores more nodes fails with GORIO_ERR_CAPACITY.
- *   warps_per_block / blocks_per_sm  launch geometry of the persistent kernel.
+ *   warps_per_block / blocks_per_sm  launch geometry of the persistent kernel (<= 24 warps).
+ *   stash_entries    per-query adjacency stash (exact navigation): entries of a direct-mapped
+ *                    table that keeps a scored node's neighbour list so that expanding it later
+ *                    needs no page; 0 = default 1024, 1 = off, else a power of two >= 64.
+ *                    It never changes results, only how many pages are waited for.
  */
 typedef struct {
   uint32_t max_inflight;
   uint32_t visited_capacity;
   uint32_t warps_per_block;
   uint32_t blocks_per_sm;
+  uint32_t stash_entries;
+  uint32_t reserved;
 } gorio_tuning;
 
 /*
@@ -139,7 +145,7 @@ typedef struct {
   /* where the worker warps' time went, ns summed over warps: serving arrived pages,
      running query phases, idle; the number of arrival-queue items consumed; ns executing copy commands */
   uint64_t warp_ns_arrivals, warp_ns_queries, warp_ns_idle, arrivals_consumed;
-  uint64_t warp_ns_copies, reserved2;
+  uint64_t warp_ns_copies, stash_hits;   /* expansions served from the adjacency stash */
 } gorio_stats_t;
 
 /* Open an index on CUDA device `cuda_device`.  *out is set only on GORIO_OK. */

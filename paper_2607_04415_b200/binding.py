@@ -44,7 +44,8 @@ class _CacheCfg(ctypes.Structure):
 
 class _Tuning(ctypes.Structure):
     _fields_ = [("max_inflight", ctypes.c_uint32), ("visited_capacity", ctypes.c_uint32),
-                ("warps_per_block", ctypes.c_uint32), ("blocks_per_sm", ctypes.c_uint32)]
+                ("warps_per_block", ctypes.c_uint32), ("blocks_per_sm", ctypes.c_uint32),
+                ("stash_entries", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
 
 
 _STAT_FIELDS = ["pages_hit", "pages_missed", "pages_fetched", "dedupe_joins", "evictions", "retries",
@@ -52,7 +53,7 @@ _STAT_FIELDS = ["pages_hit", "pages_missed", "pages_fetched", "dedupe_joins", "e
                 "resumes", "search_ns", "proxy_batches", "posted", "proxy_service_ns", "proxy_iters",
                 "proxy_ack_wait_iters", "proxy_window_full_iters", "proxy_ring_empty_iters",
                 "proxy_outstanding_sum", "warp_ns_arrivals", "warp_ns_queries", "warp_ns_idle",
-                "arrivals_consumed", "warp_ns_copies", "reserved2"]
+                "arrivals_consumed", "warp_ns_copies", "stash_hits"]
 
 
 class Stats(ctypes.Structure):
@@ -148,8 +149,8 @@ class Index:
                         int(timeout_ms), 0, 0)
         self._check(self._lib.gorio_cache_config(self._h, ctypes.byref(cfg)))
 
-    def set_tuning(self, max_inflight=0, visited_capacity=0, warps_per_block=0, blocks_per_sm=0):
-        t = _Tuning(max_inflight, visited_capacity, warps_per_block, blocks_per_sm)
+    def set_tuning(self, max_inflight=0, visited_capacity=0, warps_per_block=0, blocks_per_sm=0, stash_entries=0):
+        t = _Tuning(max_inflight, visited_capacity, warps_per_block, blocks_per_sm, stash_entries, 0)
         self._check(self._lib.gorio_set_tuning(self._h, ctypes.byref(t)))
 
     def search(self, queries: torch.Tensor, K: int, L: int, W: int, want_counters=True, stream=None):

@@ -48,18 +48,16 @@ struct gorio_index {
   u32 *parts = nullptr, *filled = nullptr;
   CacheShared *cs = nullptr;
   u64 *want_buf = nullptr; u32 want_cap = 0;
-  u64 *cpy_buf = nullptr, *fcmd_mirror = nullptr;
+  u64 *ring_copy = nullptr;
   // host-mapped communication areas
   u64 *ring_h = nullptr; u64 *ring_d = nullptr; u32 ring_cap = 0;
-  u32 *comp_h = nullptr; u32 *comp_d = nullptr;
-  u32 *hctl_h = nullptr; u32 *hctl_d = nullptr;     // [0] completion tail, [1] abort, [2] copy-command tail
-  u64 *fcmd_h = nullptr; u64 *fcmd_d = nullptr;     // copy commands, proxy -> GPU
+  u32 *hctl_h = nullptr; u32 *hctl_d = nullptr;     // [0] completions published, [1] abort, [2] requests admitted
   u32 *fdone_h = nullptr; u32 *fdone_d = nullptr;   // copy acknowledgements, GPU -> proxy
   u64 *arr_buf = nullptr; u32 arr_cap = 0;
 
   // query state
   gorio_tuning tune{};
-  u32 qs_slots = 0, qs_L = 0, qs_W = 0, qs_WR = 0, qs_K = 0, qs_seen = 0, qs_pset = 0;
+  u32 qs_slots = 0, qs_L = 0, qs_W = 0, qs_WR = 0, qs_K = 0, qs_seen = 0, qs_pset = 0, qs_stash = 0;
   void *qs_block = nullptr;
   Ctx ctx{};
   Ctl *ctl = nullptr;
@@ -118,16 +116,14 @@ cudaError_t host_mapped(T **h, T **d, size_t count) {
 
 void free_cache(gorio_index *ix) {
   cudaFree(ix->slot_data); cudaFree(ix->ptab); cudaFree(ix->smeta); cudaFree(ix->parts); cudaFree(ix->filled); cudaFree(ix->cs);
-  cudaFree(ix->want_buf); cudaFree(ix->cpy_buf); cudaFree(ix->fcmd_mirror);
-  ix->cpy_buf = ix->fcmd_mirror = nullptr;
+  cudaFree(ix->want_buf); cudaFree(ix->ring_copy);
+  ix->ring_copy = nullptr;
   if (ix->ring_h) cudaFreeHost(ix->ring_h);
-  if (ix->comp_h) cudaFreeHost(ix->comp_h);
-  if (ix->fcmd_h) cudaFreeHost(ix->fcmd_h);
   if (ix->fdone_h) cudaFreeHost(ix->fdone_h);
-  ix->fcmd_h = ix->fcmd_d = nullptr; ix->fdone_h = ix->fdone_d = nullptr;
+  ix->fdone_h = ix->fdone_d = nullptr;
   ix->slot_data = nullptr; ix->ptab = ix->smeta = nullptr; ix->parts = ix->filled = nullptr; ix->cs = nullptr;
   ix->want_buf = nullptr;
-  ix->ring_h = ix->ring_d = nullptr; ix->comp_h = ix->comp_d = nullptr;
+  ix->ring_h = ix->ring_d = nullptr;
   ix->cache_ready = false;
 }
 
@@ -150,7 +146,7 @@ void proxy_service(gorio_index *ix) {
   const u32 max_out = ix->cfg.max_outstanding;
   const auto latency = std::chrono::nanoseconds(ix->cfg.remote_latency_ns);
   volatile u64 *ring = ix->ring_h;
-  volatile u64 *fcmd = ix->fcmd_h;
+  volatile u32 *hctl = ix->hctl_h;
   volatile u32 *fdone = ix->fdone_h;
   u32 tail = 0, ct = 0, outstanding = 0;
   std::deque<InService> inflight;
@@ -172,11 +168,11 @@ void proxy_service(gorio_index *ix) {
         ix->px_error.store(1);   // a descriptor the GPU could not have produced
         return;
       }
-      fcmd[tail & ring_mask] = e;                 // same index, same lap tag
       inflight.push_back({slot, tail, now0});
       ++tail; ++outstanding; ++admitted;
     }
     if (admitted) {
+      hctl[2] = tail;                             // requests [0, tail) may be copied now
       ++batches;
       if (outstanding > max_seen) max_seen = outstanding;
     }
@@ -194,11 +190,11 @@ void proxy_service(gorio_index *ix) {
         if (now - r.admitted < latency) break;
         if (fdone[r.idx & ring_mask] != ((r.idx >> ring_shift) % 255u) + 1u) { ++ack_wait_iters; break; }
         service_ns += (u64)std::chrono::duration_cast<std::chrono::nanoseconds>(now - r.admitted).count();
-        ix->comp_h[ct & ring_mask] = (r.slot << 8) | (((ct >> ring_shift) % 255u) + 1u);
         ++ct; ++published;
         inflight.pop_front();
       }
       if (published) {
+        hctl[0] = ct;                             // completions [0, ct) are published, in ring order
         outstanding -= published;
         fetched += published;
       }
@@ -267,11 +263,8 @@ int setup_cache(gorio_index *ix) {
   CK(cudaMalloc(&ix->filled, (size_t)ix->n_slots * 4));
   CK(cudaMalloc(&ix->cs, sizeof(CacheShared)));
   CK(cudaMalloc(&ix->want_buf, (size_t)ix->want_cap * 8));
-  CK(cudaMalloc(&ix->cpy_buf, (size_t)ix->ring_cap * 8));
-  CK(cudaMalloc(&ix->fcmd_mirror, (size_t)ix->ring_cap * 8));
+  CK(cudaMalloc(&ix->ring_copy, (size_t)ix->ring_cap * 8));
   CK(host_mapped(&ix->ring_h, &ix->ring_d, ix->ring_cap));
-  CK(host_mapped(&ix->comp_h, &ix->comp_d, ix->ring_cap));
-  CK(host_mapped(&ix->fcmd_h, &ix->fcmd_d, ix->ring_cap));
   CK(host_mapped(&ix->fdone_h, &ix->fdone_d, ix->ring_cap));
   ix->preloaded = 0;
   if (cfg.preload) {
@@ -295,7 +288,7 @@ int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W) {
   const u32 seen_cap = ix->tune.visited_capacity ? ix->tune.visited_capacity : 32768u;
   const u32 pset_cap = ix->desc.pq_m ? 4096u : seen_cap;
   if (ix->qs_block && ix->qs_slots >= slots && ix->qs_L == L && ix->qs_W == W && ix->qs_K == K &&
-      ix->qs_seen == seen_cap && ix->qs_pset == pset_cap) {
+      ix->qs_seen == seen_cap && ix->qs_pset == pset_cap && ix->qs_stash == (ix->tune.stash_entries + 1u)) {
     ix->ctx.n_qslots = slots;
     return GORIO_OK;
   }
@@ -312,6 +305,9 @@ int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W) {
   const size_t o_pool = off; off += al((size_t)slots * (K + W) * 8);
   const size_t o_seen = off; off += al((size_t)slots * seen_cap * 4);
   const size_t o_pset = off; off += al((size_t)slots * pset_cap * 4);
+  const u32 stash_cap = ix->desc.pq_m ? 0u : (ix->tune.stash_entries == 1 ? 0u : (ix->tune.stash_entries ? ix->tune.stash_entries : 1024u));
+  const size_t o_stag = off; off += al((size_t)slots * stash_cap * 4);
+  const size_t o_stash = off; off += al((size_t)slots * stash_cap * (R + 1) * 4);
   CK(cudaMalloc(&ix->qs_block, off));
   ix->runq_cap = next_pow2(2ull * slots < 64 ? 64 : 2ull * slots);
   CK(cudaMalloc(&ix->run_buf, (size_t)ix->runq_cap * 8));
@@ -323,9 +319,10 @@ int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W) {
   c.items = (u32 *)(b + o_items); c.wrec = (u32 *)(b + o_wrec); c.adj = (u32 *)(b + o_adj);
   c.adjdeg = (u32 *)(b + o_adeg); c.pool = (u64 *)(b + o_pool);
   c.seen = (u32 *)(b + o_seen); c.pset = (u32 *)(b + o_pset);
+  c.stash_tag = (u32 *)(b + o_stag); c.stash = (u32 *)(b + o_stash); c.stash_cap = stash_cap;
   c.seen_cap = seen_cap; c.pset_cap = pset_cap; c.n_qslots = slots;
   ix->qs_slots = slots; ix->qs_L = L; ix->qs_W = W; ix->qs_WR = WR; ix->qs_K = K;
-  ix->qs_seen = seen_cap; ix->qs_pset = pset_cap;
+  ix->qs_seen = seen_cap; ix->qs_pset = pset_cap; ix->qs_stash = ix->tune.stash_entries + 1u;
   return GORIO_OK;
 }
 
@@ -450,7 +447,9 @@ int gorio_set_tuning(gorio_index *ix, const gorio_tuning *t) {
   if (!ix || !t) return GORIO_ERR_INVALID_ARG;
   if (t->visited_capacity && ((t->visited_capacity & (t->visited_capacity - 1)) || t->visited_capacity < 64))
     return fail(ix, GORIO_ERR_INVALID_ARG, "visited_capacity must be a power of two >= 64");
-  if (t->warps_per_block > 32) return fail(ix, GORIO_ERR_INVALID_ARG, "warps_per_block <= 32");
+  if (t->warps_per_block > 24) return fail(ix, GORIO_ERR_INVALID_ARG, "warps_per_block <= 24");
+  if (t->stash_entries > 1 && ((t->stash_entries & (t->stash_entries - 1)) || t->stash_entries < 64))
+    return fail(ix, GORIO_ERR_INVALID_ARG, "stash_entries must be 0 (default), 1 (off) or a power of two >= 64");
   ix->tune = *t;
   return GORIO_OK;
 }
@@ -481,15 +480,13 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   c.slot_data = ix->slot_data; c.ptab = ix->ptab; c.smeta = ix->smeta; c.parts = ix->parts; c.filled = ix->filled; c.cs = ix->cs;
   c.n_slots = ix->n_slots;
   c.ring = ix->ring_d; c.ring_mask = ix->ring_cap - 1; c.ring_shift = ilog2(ix->ring_cap);
-  c.comp_ring = ix->comp_d; c.comp_mask = ix->ring_cap - 1; c.host_ctl = ix->hctl_d;
-  c.fcmd = ix->fcmd_d; c.fdone = ix->fdone_d; c.host_pages = ix->pages_dev;
+  c.ring_dev = ix->ring_copy; c.host_ctl = ix->hctl_d;
+  c.fdone = ix->fdone_d; c.host_pages = ix->pages_dev;
   c.ctl = ix->ctl;
   u32 *qh = ix->ctl->q_heads;
   c.arr = Queue{(u32 *)ix->arr_buf, ix->arr_cap - 1, qh + 0, qh + 1, (int *)(qh + 2)};
   c.run = Queue{(u32 *)ix->run_buf, ix->runq_cap - 1, qh + 3, qh + 4, (int *)(qh + 5)};
   c.want = Queue{(u32 *)ix->want_buf, ix->want_cap - 1, qh + 6, qh + 7, (int *)(qh + 8)};
-  c.cpy = Queue{(u32 *)ix->cpy_buf, ix->ring_cap - 1, qh + 9, qh + 10, (int *)(qh + 11)};
-  c.fcmd_dev = ix->fcmd_mirror;
   c.nq = nq; c.K = K; c.L = L; c.W = W; c.WR = ix->qs_WR;
   c.queries = queries_dev; c.out_ids = out_ids_dev; c.out_dists = out_dists_dev;
   c.out_pages = out_pages_distinct_dev; c.out_counters = out_counters_dev;
@@ -499,9 +496,9 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
 
   // launch geometry: leave room on every SM for the proxy's copy kernels
   const bool pq = d.pq_m != 0;
-  u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 6u : 16u);
+  u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 6u : 24u);
   if (pq) { u32 lim = (200u * 1024u) / (d.pq_m * kPqKsub * 4u); if (warps > lim) warps = lim; }
-  if (warps < 3) return fail(ix, GORIO_ERR_INVALID_ARG, "search: need at least 3 warps per block (two pollers and a worker)");
+  if (warps < 2) return fail(ix, GORIO_ERR_INVALID_ARG, "search: need at least 2 warps per block (the poller and a worker)");
   int occ = 0;
   CK(search_occupancy(d.pq_m, warps, &occ));
   if (occ < 1) return fail(ix, GORIO_ERR_INVALID_ARG, "search: launch geometry does not fit an SM");
@@ -511,14 +508,13 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
 
   // reset the host-visible rings while the proxy is idle
   std::memset(ix->ring_h, 0, (size_t)ix->ring_cap * 8);
-  std::memset(ix->fcmd_h, 0, (size_t)ix->ring_cap * 8);
   std::memset(ix->fdone_h, 0, (size_t)ix->ring_cap * 4);
-  std::memset(ix->comp_h, 0, (size_t)ix->ring_cap * 4);
   std::memset(ix->hctl_h, 0, 64 * 4);
   std::atomic_thread_fence(std::memory_order_seq_cst);
 
   CK(cudaMemsetAsync(c.seen, 0xFF, (size_t)c.n_qslots * c.seen_cap * 4, stream));
   CK(cudaMemsetAsync(c.pset, 0xFF, (size_t)c.n_qslots * c.pset_cap * 4, stream));
+  if (c.stash_cap) CK(cudaMemsetAsync(c.stash_tag, 0xFF, (size_t)c.n_qslots * c.stash_cap * 4, stream));
   CK(launch_init(c, stream));
   ix->cache_dirty = true;      // until this search ends cleanly
   proxy_start(ix);
@@ -604,7 +600,7 @@ int gorio_stats(gorio_index *ix, gorio_stats_t *out) {
   out->proxy_window_full_iters = ix->host_window_full; out->proxy_ring_empty_iters = ix->host_ring_empty;
   out->proxy_iters = ix->host_iters; out->proxy_outstanding_sum = ix->host_out_sum;
   out->warp_ns_arrivals = h.stats[S_T_ARR]; out->warp_ns_queries = h.stats[S_T_RUN]; out->warp_ns_idle = h.stats[S_T_IDLE];
-  out->arrivals_consumed = h.stats[S_N_ARR]; out->warp_ns_copies = h.stats[S_T_CPY];
+  out->arrivals_consumed = h.stats[S_N_ARR]; out->warp_ns_copies = h.stats[S_T_CPY]; out->stash_hits = h.stats[S_STASH];
   return GORIO_OK;
 }
 

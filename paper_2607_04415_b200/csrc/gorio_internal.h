@@ -32,7 +32,8 @@ struct QHdr {
   u32 list_len;
   u32 n_iter, n_expand, n_eval, sum_deg, pages_distinct;
   u32 pool_len;   // PQ mode: entries in the rerank pool
-  u32 pad[4];
+  u32 worst_lo, worst_hi;   // the list's L-th key as of the last merge (all ones until the list is full)
+  u32 pad[2];
 };
 
 // Multi-producer multi-consumer ring of u32 values in HBM (cells hold sequence << 32 | value).
@@ -48,6 +49,10 @@ struct Queue {
 struct CacheShared {
   u32 hand;
   u32 bump;
+  int copy_count;  // admitted requests whose copy nobody has taken yet
+  u32 copy_head;
+  int comp_count;  // published completions whose arrival nobody has taken yet
+  u32 comp_head;
 };
 
 // Device-resident control block.
@@ -57,14 +62,14 @@ struct Ctl {
   u32 next_query;  // next query id to admit when a slot frees
   u32 done;        // queries finished
   u32 ring_head;   // request descriptors posted
-  u32 q_heads[16]; // queue head/tail/count words: arr(0,1,2) run(3,4,5) want(6,7,8) copy(9,10,11)
+  u32 q_heads[16]; // queue head/tail/count words: arr(0,1,2) run(3,4,5) want(6,7,8)
   u32 dbg[8];      // detail of the first error
   u32 census[16];  // debug snapshot (see census())
   u64 stats[32];
 };
 
 enum StatIdx { S_HIT = 0, S_MISSED, S_JOINS, S_EVICT, S_RETRY, S_DONE, S_NEVAL, S_NEXPAND,
-               S_SUMDEG, S_NITER, S_RESUMES, S_POSTED, S_T_ARR, S_T_RUN, S_T_IDLE, S_N_ARR, S_T_CPY };
+               S_SUMDEG, S_NITER, S_RESUMES, S_POSTED, S_T_ARR, S_T_RUN, S_T_IDLE, S_N_ARR, S_T_CPY, S_STASH };
 
 // Everything the persistent kernel needs, passed by value.
 struct Ctx {
@@ -84,15 +89,12 @@ struct Ctx {
   // miss ring: host-mapped, written by the GPU, consumed by the proxy
   u64 *ring;
   u32 ring_mask, ring_shift;
-  // completions and copy commands: host-mapped, written by the proxy, read by the GPU
-  const u32 *comp_ring; // completions [slot:24][lap:8]
-  u32 comp_mask;
-  const u32 *host_ctl;  // [1] abort request
-  const u64 *fcmd;      // copy commands [page:32][slot:24][lap:8], same size as the miss ring
-  u32 *fdone;           // per-command acknowledgement (lap tag), written by the GPU
+  u64 *ring_dev;        // device copy of every posted descriptor
+  // host-mapped words written by the proxy: [0] completions published, [1] abort request,
+  // [2] requests admitted (both counts are in ring order)
+  const u32 *host_ctl;
+  u32 *fdone;           // per-request copy acknowledgement (lap tag), written by the GPU
   const u8 *host_pages; // device view of the pinned host page store
-  Queue cpy;              // indices of copy commands ready for the copier warps
-  u64 *fcmd_dev;          // device mirror of the copy-command ring
   Queue arr, run, want;   // arrivals (slots / chain continuations), runnable query slots, pages awaiting a slot
   // query state
   u32 n_qslots, nq, K, L, W, WR;
@@ -106,7 +108,9 @@ struct Ctx {
   u32 *seen;     // [n_qslots][seen_cap]
   u32 *pset;     // [n_qslots][pset_cap]
   u64 *pool;     // [n_qslots][K + W]   PQ rerank pool (sorted, <= K kept)
-  u32 seen_cap, pset_cap;
+  u32 *stash;     // [n_qslots][stash_cap][R + 1] adjacency lists kept from scoring time (exact mode)
+  u32 *stash_tag; // [n_qslots][stash_cap] node id of each stash entry (all ones = empty)
+  u32 seen_cap, pset_cap, stash_cap;
   const void *queries;
   u32 *out_ids;
   void *out_dists;

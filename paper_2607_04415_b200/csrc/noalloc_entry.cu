@@ -115,20 +115,17 @@ extern "C" int gorio_search_resident_noalloc(const gorio_index_desc *d, const vo
   c.cs = cv.take<CacheShared>(1);
   c.ptab = cv.take<u64>(n_pages); c.smeta = cv.take<u64>(n_pages);
   c.parts = cv.take<u32>(n_pages); c.filled = cv.take<u32>(n_pages);
-  // proxy rings that nothing ever writes: the pollers read zeros (device memory) and idle
+  // proxy words that nothing ever writes: the poller reads zeros (device memory) and idles
   u32 *dummy = cv.take<u32>(64);
   c.host_ctl = dummy;
-  c.comp_ring = cv.take<u32>(kNaRing); c.comp_mask = kNaRing - 1;
   c.ring = cv.take<u64>(kNaRing); c.ring_mask = kNaRing - 1; c.ring_shift = 8;
-  u64 *fcmd = cv.take<u64>(kNaRing);
-  c.fcmd = fcmd; c.fcmd_dev = cv.take<u64>(kNaRing); c.fdone = cv.take<u32>(kNaRing);
+  c.ring_dev = cv.take<u64>(kNaRing); c.fdone = cv.take<u32>(kNaRing);
   c.host_pages = (const u8 *)pages_dev;
   const u32 runq = 2 * kNaSlots, arrq = 1024, smallq = 256;
   u32 *qh = c.ctl->q_heads;
   c.arr = Queue{(u32 *)cv.take<u64>(arrq), arrq - 1, qh + 0, qh + 1, (int *)(qh + 2)};
   c.run = Queue{(u32 *)cv.take<u64>(runq), runq - 1, qh + 3, qh + 4, (int *)(qh + 5)};
   c.want = Queue{(u32 *)cv.take<u64>(smallq), smallq - 1, qh + 6, qh + 7, (int *)(qh + 8)};
-  c.cpy = Queue{(u32 *)cv.take<u64>(smallq), smallq - 1, qh + 9, qh + 10, (int *)(qh + 11)};
   c.n_qslots = slots; c.nq = nq; c.K = K; c.L = L; c.W = W; c.WR = WR;
   c.hdr = cv.take<QHdr>(slots);
   c.list = cv.take<u64>((size_t)slots * L); c.cand = cv.take<u64>((size_t)slots * WR);
@@ -136,6 +133,7 @@ extern "C" int gorio_search_resident_noalloc(const gorio_index_desc *d, const vo
   c.adj = cv.take<u32>((size_t)slots * WR); c.adjdeg = cv.take<u32>((size_t)slots * W);
   c.pool = nullptr;
   c.seen_cap = kNaVisited; c.pset_cap = kNaVisited;
+  c.stash = nullptr; c.stash_tag = nullptr; c.stash_cap = 0;    // everything is resident: no stash needed
   c.seen = cv.take<u32>((size_t)slots * kNaVisited); c.pset = cv.take<u32>((size_t)slots * kNaVisited);
   if (cv.off > kNoallocScratchBytes) return na_fail(GORIO_ERR_INTERNAL, "noalloc search: scratch layout exceeds the array");
   c.queries = queries_dev; c.out_ids = out_ids_dev; c.out_dists = out_dists_dev;

@@ -98,8 +98,8 @@ __device__ __forceinline__ void stat_add(const Ctx &c, u32 idx, u32 v) {
 // for that cell is bounded by the producer's own push.
 constexpr u32 kSpinLimit = 1u << 22;
 
-__device__ void q_push(const Ctx &c, const Queue &q, u32 v) {
-  __threadfence();   // everything written for the consumer is visible before the cell
+__device__ void q_push(const Ctx &c, const Queue &q, u32 v, bool fence = true) {
+  if (fence) __threadfence();   // everything written for the consumer is visible before the cell
   const u32 pos = atomicAdd(q.tail, 1u);
   u64 *cell = (u64 *)q.buf + (pos & q.mask);
   u32 spins = 0;
@@ -168,9 +168,12 @@ struct LaneStats { u32 hit, missed, joins, evict, retry, posted; };
 // has consumed it.  (Section 3.2: reserve a descriptor slot atomically, record page id and
 // target cache slot, publish through a ready flag -- here the lap tag inside the word.)
 __device__ __forceinline__ void post_request(const Ctx &c, u32 page, u32 slot) {
-  u32 idx = atomicAdd(&c.ctl->ring_head, 1u);
-  u32 lap = ((idx >> c.ring_shift) % 255u) + 1u;
-  st_sys_u64(c.ring + (idx & c.ring_mask), ((u64)page << 32) | ((u64)slot << 8) | lap);
+  const u32 idx = atomicAdd(&c.ctl->ring_head, 1u);
+  const u32 lap = ((idx >> c.ring_shift) % 255u) + 1u;
+  const u64 e = ((u64)page << 32) | ((u64)slot << 8) | lap;
+  st_u64(c.ring_dev + (idx & c.ring_mask), e);   // device copy: what copy and arrival tickets refer to
+  __threadfence_system();      // page word, slot label and device copy before the host can act
+  st_sys_u64(c.ring + (idx & c.ring_mask), e);
 }
 
 // Get a slot for a new page: never-used slots first, then the clock (second chance for
@@ -181,7 +184,7 @@ __device__ u32 alloc_slot(const Ctx &c, u32 hint, LaneStats &st) {
     u32 b = atomicAdd(&c.cs->bump, 1u);
     if (b < c.n_slots) return b;
   }
-  const int sweep = hint != kNil ? 8 : 48;
+  const int sweep = hint != kNil ? 2 : 48;
   for (int step = 0; step <= sweep; ++step) {
     const bool use_hint = step == sweep;
     if (use_hint && hint == kNil) break;
@@ -205,13 +208,14 @@ __device__ u32 alloc_slot(const Ctx &c, u32 hint, LaneStats &st) {
 __device__ void assign_and_post(const Ctx &c, u32 page, u32 slot, LaneStats &st) {
   const u32 gen = sm_gen(ld_u64(c.smeta + slot)) + 1u;
   st_u64(c.smeta + slot, mk_sm(page, gen, 0));
-  __threadfence();
+  // (no fence needed here: a clock sweep that sees the new label with the old page word, or
+  // the reverse, finds state != RESIDENT or a slot mismatch and moves on; everyone else
+  // learns of the slot through the descriptor, which is fenced in post_request)
   for (u32 spins = 0;; ++spins) {
     const u64 w = ld_u64(c.ptab + page);
     if (pw_state(w) != P_WANTED || spins > kSpinLimit) { raise(c, 8, 0x41, page, (u32)(w >> 32), spins); return; }
     if (atomicCAS((unsigned long long *)(c.ptab + page), w, mk_pw(P_FILLING, slot, pw_low(w))) == w) break;
   }
-  __threadfence_system();      // page word and slot label visible to whoever learns of the request
   post_request(c, page, slot);
   st.posted++;
 }
@@ -285,6 +289,9 @@ __device__ __forceinline__ u64 mk_key(u32 dist, u32 id) { return ((u64)dist << 3
 __device__ __forceinline__ u32 key_id(u64 k) { return (u32)(k & 0xFFFFFFFFull) >> 1; }
 __device__ __forceinline__ u32 key_dist(u64 k) { return (u32)(k >> 32); }
 
+constexpr u32 kStashBusy = 0xFFFFFFFEu;
+__device__ __forceinline__ u32 hash32(u32 v) { v *= 0x9E3779B1u; v ^= v >> 15; return v * 0x85EBCA77u; }
+
 // Consume item j of query slot qs from the page in `slot` (warp cooperative).
 //   PH_EVAL   : score the node, write its key into the candidate buffer.
 //   PH_EXPAND : copy the node's adjacency list into the query's buffer (PQ mode: also the
@@ -296,7 +303,26 @@ __device__ void consume_item(const Ctx &c, u32 qs, u32 j, u32 slot, u32 lane) {
   const u8 *rec = c.slot_data + (u64)slot * kPageBytes + (node % c.npp) * c.node_bytes;
   if (phase == PH_EVAL) {
     u32 d = warp_dist(c, rec, qid, lane);
-    if (lane == 0) st_u64(c.cand + (u64)qs * c.WR + j, mk_key(d, node));
+    const u64 key = mk_key(d, node);
+    if (lane == 0) st_u64(c.cand + (u64)qs * c.WR + j, key);
+    // The node's page is in hand now.  If the node can still enter the list (its key beats
+    // the list's worst as of the last merge; the worst only improves, so this errs on the
+    // safe side), keep its adjacency list in the query's stash: expanding it later then
+    // needs no page.  The stash is a direct-mapped table; a busy or overwritten entry only
+    // means that the expansion goes through the page cache as usual.
+    if (c.stash_cap && key < ld_u64((const u64 *)&h->worst_lo)) {
+      const u32 e = hash32(node) & (c.stash_cap - 1);
+      u32 *tag = c.stash_tag + (u64)qs * c.stash_cap + e;
+      u32 busy = 0;
+      if (lane == 0) busy = atomicExch(tag, kStashBusy) == kStashBusy ? 1u : 0u;
+      if (!__shfl_sync(0xffffffffu, busy, 0)) {
+        const u32 *adj = (const u32 *)(rec + c.vec_bytes);
+        u32 *dst = c.stash + ((u64)qs * c.stash_cap + e) * (c.R + 1u);
+        for (u32 i = lane; i < c.R + 1u; i += 32) st_u32(dst + i, __ldcg(adj + i));   // degree, then ids
+        __syncwarp();
+        if (lane == 0) { __threadfence(); st_u32(tag, node); }
+      }
+    }
   } else {
     const u32 *adj = (const u32 *)(rec + c.vec_bytes);
     u32 deg = __ldcg(adj);
@@ -314,8 +340,98 @@ __device__ void consume_item(const Ctx &c, u32 qs, u32 j, u32 slot, u32 lane) {
 __device__ __forceinline__ void complete_items(const Ctx &c, u32 qs, u32 n) {
   __threadfence();
   u32 old = atomicSub(&c.hdr[qs].awaiting, n);
-  if (old == n) { q_push(c, c.run, qs); stat_add(c, S_RESUMES, 1); }
+  if (old == n) { q_push(c, c.run, qs, false); stat_add(c, S_RESUMES, 1); }
   else if (old < n) raise(c, 8, 0x61, qs, old, n);
+}
+
+// Consume up to 32 items at once: lane i holds item i = (query slot, item index, cache slot) if
+// bit i of `mask` is set.  The items' metadata is fetched lane-parallel, and the vectors of
+// scoring items are loaded four items at a time before any of them is reduced, so that the
+// L2 round trips of different items overlap instead of adding up (the per-item version is
+// latency bound).  Adjacency copies (expansion items) and vectors longer than 96 words take
+// the one-at-a-time path.
+__device__ __noinline__ void consume_group(const Ctx &c, u32 mask, u32 qs, u32 j, u32 slot, u32 lane) {
+  const bool mine = (mask >> lane) & 1u;
+  u32 phase = 0, qid = 0, node = 0;
+  u64 worst = 0;
+  if (mine) {
+    const QHdr *h = c.hdr + qs;
+    phase = ld_u32(&h->phase); qid = ld_u32(&h->qid);
+    node = ld_u32(c.items + (u64)qs * c.WR + j);
+    if (c.stash_cap) worst = ld_u64((const u64 *)&h->worst_lo);
+  }
+  const u32 words = c.vec_bytes >> 2;
+  const u32 eval_mask = words <= 96u ? __ballot_sync(0xffffffffu, mine && phase == PH_EVAL) : 0u;
+  u32 dist = 0;
+  for (u32 m = eval_mask; m;) {
+    u32 src[4], a[4][3], b[4][3];
+    int ng = 0;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) { src[g] = 0; if (m) { src[g] = __ffs(m) - 1; m &= m - 1; ng = g + 1; } }
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      if (g < ng) {
+        const u32 s_qid = __shfl_sync(0xffffffffu, qid, src[g]), s_node = __shfl_sync(0xffffffffu, node, src[g]);
+        const u32 s_slot = __shfl_sync(0xffffffffu, slot, src[g]);
+        const u32 *rec = (const u32 *)(c.slot_data + (u64)s_slot * kPageBytes + (s_node % c.npp) * c.node_bytes);
+        const u32 *q = (const u32 *)((const u8 *)c.queries + (u64)s_qid * c.vec_bytes);
+#pragma unroll
+        for (int w = 0; w < 3; ++w) {
+          const u32 idx = (u32)w * 32u + lane;
+          const bool in = idx < words;
+          a[g][w] = in ? __ldcg(rec + idx) : 0u;
+          b[g][w] = in ? __ldg(q + idx) : 0u;
+        }
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      if (g < ng) {
+        u32 d;
+        if (c.dtype == 0) {
+          u32 acc = 0;
+#pragma unroll
+          for (int w = 0; w < 3; ++w) { const u32 x = __vabsdiffu4(a[g][w], b[g][w]); acc = __dp4a(x, x, acc); }
+          d = __reduce_add_sync(0xffffffffu, acc);
+        } else {
+          float acc = 0.f;
+#pragma unroll
+          for (int w = 0; w < 3; ++w) { const float x = __uint_as_float(b[g][w]) - __uint_as_float(a[g][w]); acc = fmaf(x, x, acc); }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+          d = __float_as_uint(acc);
+        }
+        if (lane == src[g]) dist = d;
+      }
+    }
+  }
+  const bool scored = (eval_mask >> lane) & 1u;
+  const u64 key = mk_key(dist, node);
+  if (scored) st_u64(c.cand + (u64)qs * c.WR + j, key);
+  // adjacency stash for candidates that can still enter the list (see consume_item)
+  for (u32 m = __ballot_sync(0xffffffffu, scored && c.stash_cap && key < worst); m; m &= m - 1) {
+    const u32 src = __ffs(m) - 1;
+    const u32 s_qs = __shfl_sync(0xffffffffu, qs, src), s_node = __shfl_sync(0xffffffffu, node, src);
+    const u32 s_slot = __shfl_sync(0xffffffffu, slot, src);
+    const u32 e = hash32(s_node) & (c.stash_cap - 1);
+    u32 *tag = c.stash_tag + (u64)s_qs * c.stash_cap + e;
+    u32 busy = 0;
+    if (lane == 0) busy = atomicExch(tag, kStashBusy) == kStashBusy ? 1u : 0u;
+    if (!__shfl_sync(0xffffffffu, busy, 0)) {
+      const u32 *adj = (const u32 *)(c.slot_data + (u64)s_slot * kPageBytes + (s_node % c.npp) * c.node_bytes + c.vec_bytes);
+      u32 *dst = c.stash + ((u64)s_qs * c.stash_cap + e) * (c.R + 1u);
+      for (u32 i = lane; i < c.R + 1u; i += 32) st_u32(dst + i, __ldcg(adj + i));
+      __syncwarp();
+      if (lane == 0) { __threadfence(); st_u32(tag, s_node); }
+    }
+  }
+  // everything else one at a time
+  for (u32 m = mask & ~eval_mask; m; m &= m - 1) {
+    const u32 src = __ffs(m) - 1;
+    consume_item(c, __shfl_sync(0xffffffffu, qs, src), __shfl_sync(0xffffffffu, j, src),
+                 __shfl_sync(0xffffffffu, slot, src), lane);
+  }
+  __syncwarp();
 }
 
 // Waiter lists can be long (every query waits on the entry page at the start), so a warp
@@ -352,13 +468,14 @@ __device__ void consume_chain(const Ctx &c, u32 slot, u32 page, u32 gen, u32 g, 
     atomicAdd(c.parts + slot, 1u);
     q_push(c, c.arr, kContFlag | cur);
   }
-  for (u32 i = 0; i < n; ++i) {
-    const u32 rec = __shfl_sync(0xffffffffu, mine, i);
-    const u32 qs = rec / c.WR, j = rec % c.WR;
-    consume_item(c, qs, j, slot, lane);
-    __threadfence();      // every lane's result stores before lane 0 counts the item done
+  {
+    const bool have = lane < n;
+    const u32 qs = have ? mine / c.WR : 0u, j = have ? mine % c.WR : 0u;
+    consume_group(c, n >= 32 ? 0xffffffffu : ((1u << n) - 1u), qs, j, slot, lane);
+    // consume_group ends with a warp barrier: every lane's result stores happen before the
+    // owner lane's fence + decrement below
+    if (have) complete_items(c, qs, 1);
     __syncwarp();
-    if (lane == 0) complete_items(c, qs, 1);
   }
   u32 last = 0;
   if (lane == 0) last = atomicSub(c.parts + slot, 1u) == 1u ? 1u : 0u;
@@ -401,7 +518,6 @@ __device__ void consume_arrival(const Ctx &c, u32 v, u32 lane) {
   if (lane == 0) {
     st_u32(c.parts + slot, 1u);
     st_u64(c.smeta + slot, m | 1ull);                      // a fresh page gets its second chance
-    __threadfence();
     const u64 old = atomicExch((unsigned long long *)(c.ptab + page), mk_pw(P_ARRIVED, slot, gen));
     if (pw_state(old) != P_FILLING || pw_slot(old) != slot) { raise(c, 8, 0x72, slot, page, (u32)(old >> 32)); bad = 1; }
     head = pw_low(old);
@@ -415,7 +531,6 @@ __device__ void consume_arrival(const Ctx &c, u32 v, u32 lane) {
 // ------------------------------------------------------------------------------------------
 // per-query exact sets (open addressing, linear probing, 0xFFFFFFFF = empty)
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ u32 hash32(u32 v) { v *= 0x9E3779B1u; v ^= v >> 15; return v * 0x85EBCA77u; }
 
 // returns 1 if v was inserted now, 0 if already present, 2 if the table is full
 __device__ u32 set_insert(u32 *tab, u32 cap, u32 v) {
@@ -448,7 +563,7 @@ __device__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
   const u32 *items = c.items + (u64)qs * c.WR;
   u32 *pset = c.pset + (u64)qs * c.pset_cap;
   LaneStats st = {0, 0, 0, 0, 0, 0};
-  u32 n_done = 0, new_pages = 0;
+  u32 n_done = 0, new_pages = 0, n_stash = 0;
 
   for (u32 base = 0; base < n; base += 32) {
     const u32 j = base + lane;
@@ -463,16 +578,36 @@ __device__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
         else if (r == 2) raise(c, 6, 0x81, qs, page);
       }
     }
+    if (c.stash_cap && phase == PH_EXPAND && c.pq_m == 0) {
+      // expansions whose adjacency list was stashed when the node was scored need no page
+      u32 e = 0, have = 0;
+      if (pending) {
+        e = hash32(node) & (c.stash_cap - 1);
+        have = ld_u32(c.stash_tag + (u64)qs * c.stash_cap + e) == node ? 1u : 0u;
+      }
+      const u32 cand_mask = __ballot_sync(0xffffffffu, have != 0u);
+      for (u32 m = cand_mask; m; m &= m - 1) {
+        const u32 src = __ffs(m) - 1;
+        const u32 sj = __shfl_sync(0xffffffffu, j, src), se = __shfl_sync(0xffffffffu, e, src);
+        const u32 *from = c.stash + ((u64)qs * c.stash_cap + se) * (c.R + 1u);
+        u32 *dst = c.adj + ((u64)qs * c.W + sj) * c.R;
+        for (u32 i = lane; i < c.R; i += 32) st_u32(dst + i, ld_u32(from + 1 + i));
+        if (lane == 0) st_u32(c.adjdeg + (u64)qs * c.W + sj, ld_u32(from));
+      }
+      if (cand_mask) {
+        __threadfence();
+        if (have && ld_u32(c.stash_tag + (u64)qs * c.stash_cap + e) == node) {   // not overwritten meanwhile
+          pending = false; n_done++; n_stash++;
+        }
+      }
+    }
     for (u32 round = 0; __any_sync(0xffffffffu, pending); ++round) {
       u32 code = LK_NONE, slot = 0, gen = 0;
       if (pending) code = page_lookup(c, page, qs * c.WR + j, slot, gen, st);
       __syncwarp();
       if (code == LK_WAIT) pending = false;
       const u32 hits = __ballot_sync(0xffffffffu, code == LK_HIT);
-      for (u32 m = hits; m; m &= m - 1) {
-        const u32 src = __ffs(m) - 1;
-        consume_item(c, qs, __shfl_sync(0xffffffffu, j, src), __shfl_sync(0xffffffffu, slot, src), lane);
-      }
+      if (hits) consume_group(c, hits, qs, j, slot, lane);
       if (hits) {
         __threadfence();
         if (code == LK_HIT) {
@@ -499,6 +634,7 @@ __device__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
   for (int o = 16; o > 0; o >>= 1) {
     n_done += __shfl_xor_sync(0xffffffffu, n_done, o);
     new_pages += __shfl_xor_sync(0xffffffffu, new_pages, o);
+    n_stash += __shfl_xor_sync(0xffffffffu, n_stash, o);
     st.hit += __shfl_xor_sync(0xffffffffu, st.hit, o);
     st.missed += __shfl_xor_sync(0xffffffffu, st.missed, o);
     st.joins += __shfl_xor_sync(0xffffffffu, st.joins, o);
@@ -512,6 +648,7 @@ __device__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
   if (lane == 0) {
     stat_add(c, S_HIT, st.hit); stat_add(c, S_MISSED, st.missed); stat_add(c, S_JOINS, st.joins);
     stat_add(c, S_EVICT, st.evict); stat_add(c, S_RETRY, st.retry); stat_add(c, S_POSTED, st.posted);
+    stat_add(c, S_STASH, n_stash);
     if (new_pages) st_u32(&h->pages_distinct, ld_u32(&h->pages_distinct) + new_pages);
     __threadfence();
     const u32 old = atomicSub(&h->awaiting, n_done + 1u);       // inline hits and the guard
@@ -616,6 +753,14 @@ __device__ __noinline__ u32 merge_select(const Ctx &c, u32 qs, u32 lane) {
     if (e < len) st_u64(list + e, x[r]);
   }
   if (lane == 0) st_u32(&h->list_len, len);
+  {   // the L-th key once the list is full: what a new candidate has to beat
+    const u32 wi = c.L - 1u;
+    u64 worst = kPadKey;
+#pragma unroll
+    for (int r = 0; r < NPL; ++r)
+      if ((u32)r == wi / 32u) worst = __shfl_sync(0xffffffffu, x[r], wi % 32u);
+    if (lane == 0) st_u64((u64 *)&h->worst_lo, len == c.L ? (worst | 1ull) : kPadKey);
+  }
   if (taken == 0 && c.pq_m == 0) {
     const u32 qid = uld(&h->qid);
 #pragma unroll
@@ -775,6 +920,7 @@ __device__ __forceinline__ void reset_hdr(QHdr *h, u32 qid) {
   st_u32(&h->qid, qid); st_u32(&h->phase, PH_NEW); st_u32(&h->awaiting, 0); st_u32(&h->n_items, 0);
   st_u32(&h->reserved0, 0); st_u32(&h->list_len, 0); st_u32(&h->n_iter, 0); st_u32(&h->n_expand, 0);
   st_u32(&h->n_eval, 0); st_u32(&h->sum_deg, 0); st_u32(&h->pages_distinct, 0); st_u32(&h->pool_len, 0);
+  st_u32(&h->worst_lo, 0xFFFFFFFFu); st_u32(&h->worst_hi, 0xFFFFFFFFu);
 }
 
 // The slot's query is done: admit the next unstarted query into the same slot, if any.
@@ -788,6 +934,8 @@ __device__ bool recycle_slot(const Ctx &c, u32 qs, u32 lane) {
   for (u32 i = lane; i < c.seen_cap / 4; i += 32) __stcg(s4 + i, ff);
   uint4 *p4 = (uint4 *)(c.pset + (u64)qs * c.pset_cap);
   for (u32 i = lane; i < c.pset_cap / 4; i += 32) __stcg(p4 + i, ff);
+  uint4 *t4 = (uint4 *)(c.stash_tag + (u64)qs * c.stash_cap);
+  for (u32 i = lane; i < c.stash_cap / 4; i += 32) __stcg(t4 + i, ff);
   if (lane == 0) reset_hdr(c.hdr + qs, nxt);
   __threadfence();
   __syncwarp();
@@ -856,14 +1004,15 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut) {
   if (lane == 0) raise(c, 6, 0xA2, qs);
 }
 
-// Execute one of the proxy's copy commands (mirrored into device memory by the poller): pull
+// Execute the copy of admitted request idx (the proxy admits requests in ring order and
+// publishes how many; the request itself is read from the device copy of the ring): pull
 // the 4 KB page from the pinned store into its cache slot.  Any worker warp does this, ahead
 // of all other work; only the page bytes cross the host link on this path.  The host is told
 // as soon as the page's bytes have arrived on the GPU (they are in registers), so that no
 // fence sits inside the proxy's outstanding window; the stores into the slot are then
 // released to the consumers of the arrival through the slot's `filled` generation.
 __device__ void copy_page(const Ctx &c, u32 idx, u32 lane) {
-  const u64 cmd = __shfl_sync(0xffffffffu, ld_u64(c.fcmd_dev + (idx & c.ring_mask)), 0);
+  const u64 cmd = __shfl_sync(0xffffffffu, ld_u64(c.ring_dev + (idx & c.ring_mask)), 0);
   const u32 page = (u32)(cmd >> 32), slot = (u32)(cmd >> 8) & 0xFFFFFFu;
   if (page >= c.n_pages || slot >= c.n_slots) { if (lane == 0) raise(c, 8, 0xC1, idx, page, slot); return; }
   const uint4 *src = (const uint4 *)(c.host_pages + (u64)page * kPageBytes);
@@ -885,31 +1034,6 @@ __device__ void copy_page(const Ctx &c, u32 idx, u32 lane) {
     __threadfence();
     st_u32(c.filled + slot, gen);
   }
-}
-
-// Push n values with one ticket reservation and one count update for the whole warp: value k
-// of this lane goes to position ofs[k] (0 <= ofs < n, all distinct) if take[k].
-template <int NV>
-__device__ __forceinline__ void bulk_push(const Ctx &c, const Queue &q, const u32 (&val)[NV], const u32 (&ofs)[NV],
-                                          const bool (&take)[NV], u32 n, u32 lane) {
-  if (n == 0) return;
-  u32 base = 0;
-  if (lane == 0) { __threadfence(); base = atomicAdd(q.tail, n); }
-  base = __shfl_sync(0xffffffffu, base, 0);
-#pragma unroll
-  for (int k = 0; k < NV; ++k) {
-    if (take[k]) {
-      const u32 pos = base + ofs[k];
-      u64 *cell = (u64 *)q.buf + (pos & q.mask);
-      u32 spins = 0;
-      while ((u32)(ld_u64(cell) >> 32) != pos) {
-        if (++spins > kSpinLimit) { raise(c, 8, 0x53, pos); break; }
-      }
-      st_u64(cell, ((u64)(pos + 1u) << 32) | val[k]);
-    }
-  }
-  __syncwarp();
-  if (lane == 0) atomicAdd(q.count, (int)n);
 }
 
 // Debug aid: one snapshot of where slots, pages and queries are, taken by the poller warp.
@@ -936,80 +1060,52 @@ __device__ void census(const Ctx &c, u32 lane) {
   for (int i = 0; i < 12; ++i) cnt[i] = __reduce_add_sync(0xffffffffu, cnt[i]);
   if (lane == 0) {
     for (int i = 0; i < 9; ++i) c.ctl->census[i] = cnt[i];
-    c.ctl->census[9] = (u32)*c.want.count; c.ctl->census[10] = (u32)*c.arr.count; c.ctl->census[11] = (u32)*c.run.count;
+    c.ctl->census[9] = (u32)*c.want.count; c.ctl->census[10] = (u32)c.cs->comp_count; c.ctl->census[11] = (u32)*c.run.count;
     c.ctl->census[12] = ld_u32(&c.ctl->done); c.ctl->census[13] = ld_u32(&c.ctl->ring_head);
   }
 }
 
-// Two poller warps are the only warps that read control data from host memory: warp 0 of
-// block 0 follows the proxy's completion ring, warp 0 of block 1 (or warp 1 of block 0 in a
-// one-block launch) its copy-command ring.  Ring entries are self-validating through a lap
-// tag, so per iteration a poller reads the next 256 ring positions with fully coalesced
-// 512-byte warp loads and forwards the valid prefix in bulk: completions to the arrival
-// queue; commands, mirrored into device memory, to the copy queue.  The abort word is
-// sampled now and then.
-constexpr u32 kPollWidth = 256;
-
-__device__ void poller(const Ctx &c, bool commands, u32 lane) {
-  u32 seen = 0, it = 0;
+// Warp 0 of block 0 is the only warp that reads control words from host memory.  The proxy
+// admits requests and publishes completions in ring order, and the GPU keeps its own copy of
+// every descriptor, so all the host has to say is two counters: how many requests are
+// admitted (their pages may be copied now) and how many completions are published (their
+// pages have "arrived").  One 16-byte read per iteration fetches both and the abort word;
+// the poller turns the deltas into tickets that worker warps take with fetch-and-add.
+__device__ void poller(const Ctx &c, u32 lane) {
+  u32 seen_pub = 0, seen_adm = 0, it = 0;
   const u64 t0 = globaltimer();
-  bool census_done = c.census_ns == 0 || commands;
+  bool census_done = c.census_ns == 0;
   for (;;) {
     if (warp_stopped(c)) break;
     if (!census_done && globaltimer() - t0 > c.census_ns) { census(c, lane); census_done = true; }
-    const u32 base = seen & ~7u;        // 8 | base keeps every 16-byte load inside the ring
-    u32 val[8], rel[8]; bool take[8]; u32 first_bad = kPollWidth;
-    u64 w[8];
-    if (!commands) {
-      // load k covers ring positions base + 128k + [0,128): lane l gets 4 of them
-      uint4 q4[2];
-#pragma unroll
-      for (int k = 0; k < 2; ++k) q4[k] = ld_sys_v4(c.comp_ring + ((base + 128u * k + 4u * lane) & c.comp_mask));
-#pragma unroll
-      for (int k = 0; k < 2; ++k) {
-        const u32 e[4] = {q4[k].x, q4[k].y, q4[k].z, q4[k].w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) { rel[4 * k + j] = 128u * k + 4u * lane + j; val[4 * k + j] = e[j] >> 8; w[4 * k + j] = e[j]; }
-      }
-    } else {
-      // load k covers ring positions base + 64k + [0,64): lane l gets 2 of them
-      uint4 q4[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) q4[k] = ld_sys_v4((const u32 *)(c.fcmd + ((base + 64u * k + 2u * lane) & c.ring_mask)));
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        w[2 * k] = ((u64)q4[k].y << 32) | q4[k].x; w[2 * k + 1] = ((u64)q4[k].w << 32) | q4[k].z;
-        rel[2 * k] = 64u * k + 2u * lane; rel[2 * k + 1] = rel[2 * k] + 1u;
-      }
+    u32 pub = 0, abort_req = 0, adm = 0;
+    if (lane == 0) {
+      const uint4 h = ld_sys_v4(c.host_ctl);
+      pub = h.x; abort_req = h.y; adm = h.z;
+      if (adm != seen_adm) atomicAdd(&c.cs->copy_count, (int)(adm - seen_adm));
+      if (pub != seen_pub) atomicAdd(&c.cs->comp_count, (int)(pub - seen_pub));
+      if (adm == seen_adm && pub == seen_pub) __nanosleep(100);
+      seen_adm = adm; seen_pub = pub;
     }
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const u32 i = base + rel[k];
-      const bool ok = ((u32)w[k] & 0xFFu) == ((i >> c.ring_shift) % 255u) + 1u || i < seen;
-      if (!ok && rel[k] < first_bad) first_bad = rel[k];
-    }
-    const u32 end = base + __reduce_min_sync(0xffffffffu, first_bad);   // [seen, end) new and valid
-    u32 ofs[8];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const u32 i = base + rel[k];
-      take[k] = i >= seen && i < end;
-      ofs[k] = i - seen;
-      if (commands) { val[k] = i; if (take[k]) st_u64(c.fcmd_dev + (i & c.ring_mask), w[k]); }
-    }
-    bulk_push<8>(c, commands ? c.cpy : c.arr, val, ofs, take, end - seen, lane);
-    if (end == seen) __nanosleep(100);
-    seen = end;
-    if ((++it & 15u) == 0) {
-      u32 abort_req = 0, late = 0;
-      if (lane == 0) {
-        abort_req = ld_sys_u32(c.host_ctl + 1);
-        late = globaltimer() - t0 > c.timeout_ns ? 1u : 0u;
-      }
-      if (__shfl_sync(0xffffffffu, abort_req, 0)) { if (lane == 0) raise(c, 5, 0xB1); break; }
-      if (__shfl_sync(0xffffffffu, late, 0)) { if (lane == 0) raise(c, 5, 0xB2); break; }
-    }
+    abort_req = __shfl_sync(0xffffffffu, abort_req, 0);
+    if (abort_req) { if (lane == 0) raise(c, 5, 0xB1); break; }
+    u32 late = ((++it & 63u) == 0 && globaltimer() - t0 > c.timeout_ns) ? 1u : 0u;
+    if (__shfl_sync(0xffffffffu, late, 0)) { if (lane == 0) raise(c, 5, 0xB2); break; }
   }
+}
+
+// Take one ticket from a (count, head) pair released by the poller; lane 0 only.
+__device__ __forceinline__ bool take_ticket(int *count, u32 *head, u32 &idx) {
+  if ((int)ld_u32((const u32 *)count) <= 0) return false;
+  if (atomicSub(count, 1) <= 0) { atomicAdd(count, 1); return false; }
+  idx = atomicAdd(head, 1u);
+  return true;
+}
+__device__ __forceinline__ bool warp_ticket(int *count, u32 *head, u32 &idx, u32 lane) {
+  u32 ok = 0, v = 0;
+  if (lane == 0) ok = take_ticket(count, head, v) ? 1u : 0u;
+  idx = __shfl_sync(0xffffffffu, v, 0);
+  return __shfl_sync(0xffffffffu, ok, 0) != 0u;
 }
 
 // Register budget: at most 80 per thread, so that 20 resident warps leave register file and
@@ -1018,8 +1114,7 @@ template <bool PQ>
 __global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
   extern __shared__ u32 smem_lut[];
   const u32 lane = lane_id(), warp = threadIdx.x >> 5;
-  if (blockIdx.x == 0 && warp == 0) { poller(c, false, lane); return; }
-  if ((gridDim.x > 1 && blockIdx.x == 1 && warp == 0) || (gridDim.x == 1 && warp == 1)) { poller(c, true, lane); return; }
+  if (blockIdx.x == 0 && warp == 0) { poller(c, lane); return; }
   u32 *lut = PQ ? smem_lut + (u64)warp * c.pq_m * kPqKsub : nullptr;
   const u64 t0 = globaltimer();
   u32 idle = 0;
@@ -1029,12 +1124,18 @@ __global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
   for (;;) {
     if (warp_stopped(c)) break;
     u32 v;
-    if (warp_pop(c, c.cpy, v, lane)) {           // the outstanding window waits on these
+    if (warp_ticket(&c.cs->copy_count, &c.cs->copy_head, v, lane)) {   // the outstanding window waits on these
       copy_page(c, v, lane); idle = 0;
       const u64 t = globaltimer(); t_cpy += t - tp; tp = t;
       continue;
     }
-    if (warp_pop(c, c.arr, v, lane)) {
+    if (warp_ticket(&c.cs->comp_count, &c.cs->comp_head, v, lane)) {   // completion v: its page has arrived
+      const u64 e = __shfl_sync(0xffffffffu, ld_u64(c.ring_dev + (v & c.ring_mask)), 0);
+      consume_arrival(c, (u32)(e >> 8) & 0xFFFFFFu, lane); idle = 0;
+      const u64 t = globaltimer(); t_arr += t - tp; tp = t; ++n_arr;
+      continue;
+    }
+    if (warp_pop(c, c.arr, v, lane)) {             // handed-off waiter chains
       consume_arrival(c, v, lane); idle = 0;
       const u64 t = globaltimer(); t_arr += t - tp; tp = t; ++n_arr;
       continue;
@@ -1072,8 +1173,7 @@ __global__ void init_kernel(const Ctx c) {
   const u32 tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
   for (u32 i = tid; i < c.n_qslots; i += nth) reset_hdr(c.hdr + i, i);
   // runnable queue starts with every slot; the others start empty
-  u64 *run = (u64 *)c.run.buf, *arr = (u64 *)c.arr.buf, *want = (u64 *)c.want.buf, *cpy = (u64 *)c.cpy.buf;
-  for (u32 i = tid; i <= c.cpy.mask; i += nth) cpy[i] = (u64)i << 32;
+  u64 *run = (u64 *)c.run.buf, *arr = (u64 *)c.arr.buf, *want = (u64 *)c.want.buf;
   for (u32 i = tid; i <= c.run.mask; i += nth) run[i] = i < c.n_qslots ? (((u64)(i + 1u) << 32) | i) : ((u64)i << 32);
   for (u32 i = tid; i <= c.arr.mask; i += nth) arr[i] = (u64)i << 32;
   for (u32 i = tid; i <= c.want.mask; i += nth) want[i] = (u64)i << 32;
@@ -1084,6 +1184,7 @@ __global__ void init_kernel(const Ctx c) {
     for (int i = 0; i < 8; ++i) ctl->dbg[i] = 0;
     *c.run.tail = c.n_qslots;
     *c.run.count = (int)c.n_qslots;
+    c.cs->copy_count = 0; c.cs->copy_head = 0; c.cs->comp_count = 0; c.cs->comp_head = 0;
   }
 }
 
