@@ -305,7 +305,11 @@ int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W) {
   const size_t o_pool = off; off += al((size_t)slots * (K + W) * 8);
   const size_t o_seen = off; off += al((size_t)slots * seen_cap * 4);
   const size_t o_pset = off; off += al((size_t)slots * pset_cap * 4);
-  const u32 stash_cap = ix->desc.pq_m ? 0u : (ix->tune.stash_entries == 1 ? 0u : (ix->tune.stash_entries ? ix->tune.stash_entries : 1024u));
+  // adjacency stash: exact navigation only; by default on (1024 entries) unless every page has
+  // a slot of its own, in which case expansions seldom wait for a page and the copies are waste
+  u32 stash_cap = ix->tune.stash_entries > 1 ? ix->tune.stash_entries
+                  : (ix->tune.stash_entries == 1 || ix->n_slots >= ix->n_pages ? 0u : 1024u);
+  if (ix->desc.pq_m) stash_cap = 0;
   const size_t o_stag = off; off += al((size_t)slots * stash_cap * 4);
   const size_t o_stash = off; off += al((size_t)slots * stash_cap * (R + 1) * 4);
   CK(cudaMalloc(&ix->qs_block, off));
@@ -496,7 +500,15 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
 
   // launch geometry: leave room on every SM for the proxy's copy kernels
   const bool pq = d.pq_m != 0;
-  u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 6u : 24u);
+  // default warps per SM: 24 when pages will be missed (arrivals are served by whoever is free);
+  // with every page resident one warp carries one query at a time, so no more than there are
+  // queries per SM (fewer idle warps polling the queues), within 8..24
+  u32 auto_warps = 24u;
+  if (ix->n_slots >= ix->n_pages) {
+    auto_warps = (nq + (u32)ix->n_sms - 1) / (u32)ix->n_sms;
+    auto_warps = auto_warps < 8u ? 8u : (auto_warps > 24u ? 24u : auto_warps);
+  }
+  u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 6u : auto_warps);
   if (pq) { u32 lim = (200u * 1024u) / (d.pq_m * kPqKsub * 4u); if (warps > lim) warps = lim; }
   if (warps < 2) return fail(ix, GORIO_ERR_INVALID_ARG, "search: need at least 2 warps per block (the poller and a worker)");
   int occ = 0;
