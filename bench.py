@@ -89,10 +89,10 @@ def l2_flush(buf):
     buf.add_(1)          # 512 MB read+write, larger than the 126 MB L2
 
 
-def oracle_qps(w, threads, budget_s=20.0):
+def oracle_qps(w, threads, budget_s=20.0, use_pq=False):
     """The CPU oracle as it stands on a bounded sample of the same queries."""
     from oracle import OracleIndex
-    orc = OracleIndex.from_workload(w)
+    orc = OracleIndex.from_workload(w, use_pq=use_pq)
     t = time.perf_counter(); orc.search(w.queries[: 4 * threads], w.K, w.L, w.W, threads=threads)
     per_q = (time.perf_counter() - t) / (4 * threads)
     n = int(min(w.nq, max(8 * threads, budget_s / max(per_q, 1e-6))))
@@ -110,7 +110,14 @@ def main():
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the index (profiling captures only)")
     ap.add_argument("--cache-frac", type=float, default=0.20)
     ap.add_argument("--preload", action="store_true", help="fully resident cache (profiling captures only)")
-    ap.add_argument("--nq", type=int, default=10_000)
+    ap.add_argument("--nq", type=int, default=None)
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5],
+                    help="3 = the benchmark workload; the others are the parity configurations")
+    ap.add_argument("--blocking", action="store_true", help="ablation: warps wait in place on a miss")
+    ap.add_argument("--latency-us", type=float, default=None)
+    ap.add_argument("--max-outstanding", type=int, default=None)
+    ap.add_argument("--L", type=int, default=None)
+    ap.add_argument("--W", type=int, default=None)
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -123,14 +130,14 @@ def main():
     if args.impl == "reference":
         if rank != 0:
             return
-        w = make_config(3, scale=args.scale, nq=args.nq, device="cuda" if torch.cuda.is_available() else "cpu",
+        w = make_config(args.config, scale=args.scale, nq=args.nq, device="cuda" if torch.cuda.is_available() else "cpu",
                         with_gt=False)
         vals = []
         for _ in range(args.warmup):
-            oracle_qps(w, threads, budget_s=2.0)
+            oracle_qps(w, threads, budget_s=2.0, use_pq=args.config == 4)
         n_s = 0
         for _ in range(args.steps):
-            v, n_s = oracle_qps(w, threads, budget_s=max(5.0, 60.0 / max(1, args.steps)))
+            v, n_s = oracle_qps(w, threads, budget_s=max(5.0, 60.0 / max(1, args.steps)), use_pq=args.config == 4)
             vals.append(v)
         v = statistics.mean(vals)
         sample = f"first {n_s} of {w.nq} queries per step, {threads} threads, in-memory page store, no cache emulation"
@@ -138,7 +145,7 @@ def main():
             "impl": "reference", "metric": METRIC, "value": v, "unit": "queries/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * n_s / v, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-            "config": {"workload": f"cfg3 SIFT1M-shaped: N={w.N} d=128 u8 R=64 npp=10 K=10 L=100 W=4"},
+            "config": {"workload": f"cfg{args.config}: N={w.N} d={w.d} {w.dtype} R={w.R} npp={w.npp} K={w.K} L={w.L} W={w.W}"},
             "cpu_baseline": {"value": v, "unit": "queries/s", "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": v, "unit": "queries/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         }))
@@ -161,14 +168,26 @@ def main():
         torch.cuda.synchronize()
 
     # every rank searches its own 10,000 queries (weak scaling): query seed 1 + rank
-    w = make_config(3, scale=args.scale, nq=args.nq, device=dev, seed_q=1 + rank)
-    cap = w.n_pages if args.preload else int(args.cache_frac * w.n_pages)
-    lat_ns, max_out = 20_000, 256
-    ix = g.Index.from_workload(w, device=local)
+    w = make_config(args.config, scale=args.scale, nq=args.nq, device=dev, seed_q=1 + rank)
+    if args.L:
+        w.L = args.L
+    if args.W:
+        w.W = args.W
+    frac = args.cache_frac if args.config in (3, 4) else w.cache_frac
+    preload = args.preload or w.preload or frac >= 1.0
+    cap = w.n_pages if preload else int(frac * w.n_pages)
+    if args.latency_us is not None:
+        w.latency_us = args.latency_us
+    if args.max_outstanding:
+        w.max_outstanding = args.max_outstanding
+    lat_ns, max_out = int(w.latency_us * 1000), w.max_outstanding
+    ix = g.Index.from_workload(w, device=local, use_pq=(args.config == 4))
+    if args.blocking:
+        ix.set_tuning(blocking=1)
     q_dev = torch.as_tensor(w.queries).to(dev)
     q_pin = torch.as_tensor(w.queries).pin_memory()
     outs_pin = dict(ids=torch.empty((w.nq, w.K), dtype=torch.int32).pin_memory(),
-                    dists=torch.empty((w.nq, w.K), dtype=torch.int32).pin_memory(),
+                    dists=torch.empty((w.nq, w.K), dtype=torch.int32 if w.dtype == "u8" else torch.float32).pin_memory(),
                     pages=torch.empty(w.nq, dtype=torch.int32).pin_memory(),
                     counters=torch.empty((w.nq, 5), dtype=torch.int32).pin_memory())
     flush = torch.zeros(512 << 20, dtype=torch.uint8, device=dev)
@@ -176,7 +195,7 @@ def main():
     pk, pk_kind = peaks()
 
     def reset_cache():
-        ix.cache_config(cap, remote_latency_ns=lat_ns, max_outstanding=max_out, preload=args.preload,
+        ix.cache_config(cap, remote_latency_ns=lat_ns, max_outstanding=max_out, preload=preload,
                         timeout_ms=120_000)
         ix.stats_reset()
         l2_flush(flush)
@@ -223,7 +242,11 @@ def main():
 
     # roofline: the slowest of (a) algorithmic HBM bytes at the measured copy peak, (b) fetched
     # page bytes over the measured host link, (c) outstanding window / injected latency
-    b_alg = st["n_eval"] * w.d + 4 * st["n_expand"] + 4 * st["sum_degree"]
+    esz = 1 if w.dtype == "u8" else 4
+    if args.config == 4:      # PQ: 32-byte code per scored node, whole record per expanded node
+        b_alg = st["n_eval"] * 32 + st["n_expand"] * w.node_bytes
+    else:
+        b_alg = st["n_eval"] * w.d * esz + 4 * st["n_expand"] + 4 * st["sum_degree"]
     b_hbm = b_alg + 4096 * fetched
     t_a = b_hbm / (pk["hbm_gbs"] * 1e9)
     t_b = 4096 * fetched / (h2d * 1e9)
@@ -236,16 +259,18 @@ def main():
     elif bound == "host_link":
         ach, peak, unit = 4096 * fetched / (ms * 1e-3) / 1e9, h2d, "GB/s"
     else:
-        ach, peak, unit = fetched / (ms * 1e-3) / 1e6, max_out / (lat_ns * 1e-9) / 1e6, "Mfetch/s"
+        ach, peak, unit = fetched / (ms * 1e-3) / 1e6, max_out / max(lat_ns * 1e-9, 1e-12) / 1e6, "Mfetch/s"
 
     ids = out["ids"].cpu().numpy().view(np.uint32)
     recall = recall_at_k(ids, w.gt)
     line = {
         "metric": METRIC, "value": world * w.nq / (ms * 1e-3), "unit": "queries/s", "n_gpus": world,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": f"cfg3 SIFT1M-shaped: N={w.N} d=128 u8 R=64 npp=10 pages={w.n_pages} "
-                               f"nq={w.nq}/gpu K=10 L=100 W=4 cache={cap} slots cold latency=20us max_outstanding=256",
+        "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": f"cfg{args.config}{' SIFT1M-shaped' if args.config == 3 else ''}: N={w.N} d={w.d} {w.dtype} "
+                               f"R={w.R} npp={w.npp} pages={w.n_pages} nq={w.nq}/gpu K={w.K} L={w.L} W={w.W} "
+                               f"cache={cap} slots {'preloaded' if preload else 'cold'} latency={w.latency_us:g}us "
+                               f"max_outstanding={max_out}{' PQ 32x256' if args.config == 4 else ''}{' BLOCKING ablation' if args.blocking else ''}",
                    "recall_at_10": recall, "l2": "flushed before every step (512 MB read+write)",
                    "cache": "re-created cold before every step, untimed", "parallelism": f"query-sharded x{world}",
                    "context": PAPER_CONTEXT},
@@ -266,7 +291,7 @@ def main():
                                      "warp_ns_queries", "warp_ns_idle", "arrivals_consumed")},
     }
     if rank == 0 and world == 1:
-        v, n_s = oracle_qps(w, threads)
+        v, n_s = oracle_qps(w, threads, use_pq=args.config == 4)
         line["cpu_baseline"] = {"value": v, "unit": "queries/s", "cores": threads, "kind": "oracle",
                                 "sample": f"first {n_s} of {w.nq} queries, {threads} threads, in-memory page store "
                                           "(no cache emulation, no injected latency)"}

@@ -109,6 +109,9 @@ typedef struct {
  *                    table that keeps a scored node's neighbour list so that expanding it later
  *                    needs no page; 0 = default 1024, 1 = off, else a power of two >= 64.
  *                    It never changes results, only how many pages are waited for.
+ *   blocking         1 = ablation: a warp that misses keeps its query and waits in place for
+ *                    the pages (the demand-paging baseline of Section 5.1) instead of parking
+ *                    the query and taking another; results are identical, only slower.
  */
 typedef struct {
   uint32_t max_inflight;
@@ -116,7 +119,7 @@ typedef struct {
   uint32_t warps_per_block;
   uint32_t blocks_per_sm;
   uint32_t stash_entries;
-  uint32_t reserved;
+  uint32_t blocking;
 } gorio_tuning;
 
 /*

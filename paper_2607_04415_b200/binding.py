@@ -45,7 +45,7 @@ class _CacheCfg(ctypes.Structure):
 class _Tuning(ctypes.Structure):
     _fields_ = [("max_inflight", ctypes.c_uint32), ("visited_capacity", ctypes.c_uint32),
                 ("warps_per_block", ctypes.c_uint32), ("blocks_per_sm", ctypes.c_uint32),
-                ("stash_entries", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+                ("stash_entries", ctypes.c_uint32), ("blocking", ctypes.c_uint32)]
 
 
 _STAT_FIELDS = ["pages_hit", "pages_missed", "pages_fetched", "dedupe_joins", "evictions", "retries",
@@ -64,7 +64,8 @@ class Stats(ctypes.Structure):
 
 
 def lib_path() -> str:
-    return os.path.join(_HERE, "libgorio.so")
+    """libgorio.so next to this file, or the build named by $GORIO_LIB (to compare two builds)."""
+    return os.environ.get("GORIO_LIB") or os.path.join(_HERE, "libgorio.so")
 
 
 def load_library():
@@ -149,8 +150,9 @@ class Index:
                         int(timeout_ms), 0, 0)
         self._check(self._lib.gorio_cache_config(self._h, ctypes.byref(cfg)))
 
-    def set_tuning(self, max_inflight=0, visited_capacity=0, warps_per_block=0, blocks_per_sm=0, stash_entries=0):
-        t = _Tuning(max_inflight, visited_capacity, warps_per_block, blocks_per_sm, stash_entries, 0)
+    def set_tuning(self, max_inflight=0, visited_capacity=0, warps_per_block=0, blocks_per_sm=0, stash_entries=0,
+                   blocking=0):
+        t = _Tuning(max_inflight, visited_capacity, warps_per_block, blocks_per_sm, stash_entries, int(blocking))
         self._check(self._lib.gorio_set_tuning(self._h, ctypes.byref(t)))
 
     def search(self, queries: torch.Tensor, K: int, L: int, W: int, want_counters=True, stream=None):

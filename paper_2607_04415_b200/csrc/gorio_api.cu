@@ -488,14 +488,16 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   c.fdone = ix->fdone_d; c.host_pages = ix->pages_dev;
   c.ctl = ix->ctl;
   u32 *qh = ix->ctl->q_heads;
-  c.arr = Queue{(u32 *)ix->arr_buf, ix->arr_cap - 1, qh + 0, qh + 1, (int *)(qh + 2)};
-  c.run = Queue{(u32 *)ix->run_buf, ix->runq_cap - 1, qh + 3, qh + 4, (int *)(qh + 5)};
-  c.want = Queue{(u32 *)ix->want_buf, ix->want_cap - 1, qh + 6, qh + 7, (int *)(qh + 8)};
+  int *cnt = ix->ctl->counts;
+  c.arr = Queue{(u32 *)ix->arr_buf, ix->arr_cap - 1, qh + 0, qh + 1, cnt + 2};
+  c.run = Queue{(u32 *)ix->run_buf, ix->runq_cap - 1, qh + 3, qh + 4, cnt + 3};
+  c.want = Queue{(u32 *)ix->want_buf, ix->want_cap - 1, qh + 6, qh + 7, cnt + 4};
   c.nq = nq; c.K = K; c.L = L; c.W = W; c.WR = ix->qs_WR;
   c.queries = queries_dev; c.out_ids = out_ids_dev; c.out_dists = out_dists_dev;
   c.out_pages = out_pages_distinct_dev; c.out_counters = out_counters_dev;
   c.timeout_ns = (u64)ix->cfg.timeout_ms * 1000000ull;
   c.max_iters = 64u * L + 1024u;
+  c.blocking = ix->tune.blocking ? 1u : 0u;
   { const char *e = std::getenv("GORIO_CENSUS_MS"); c.census_ns = e ? (u64)std::atof(e) * 1000000ull : 0; }
 
   // launch geometry: leave room on every SM for the proxy's copy kernels

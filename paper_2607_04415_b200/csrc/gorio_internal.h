@@ -49,20 +49,22 @@ struct Queue {
 struct CacheShared {
   u32 hand;
   u32 bump;
-  int copy_count;  // admitted requests whose copy nobody has taken yet
-  u32 copy_head;
-  int comp_count;  // published completions whose arrival nobody has taken yet
-  u32 comp_head;
+  u32 copy_head;   // next admitted request to copy
+  u32 comp_head;   // next published completion to consume
 };
 
 // Device-resident control block.
 struct Ctl {
+  // work counters, together in one 32-byte sector so that an idle warp reads them at once:
+  // [0] admitted requests nobody copies yet, [1] published completions nobody consumes yet,
+  // [2] arrival queue, [3] runnable queue, [4] want queue (items pushed minus items claimed)
+  int counts[8];
   u32 stop;        // 0 run, 1 all queries done, 2 error/abort
   u32 status;      // first gorio_status raised on the device
   u32 next_query;  // next query id to admit when a slot frees
   u32 done;        // queries finished
   u32 ring_head;   // request descriptors posted
-  u32 q_heads[16]; // queue head/tail/count words: arr(0,1,2) run(3,4,5) want(6,7,8)
+  u32 q_heads[16]; // queue head/tail words: arr(0,1) run(3,4) want(6,7)
   u32 dbg[8];      // detail of the first error
   u32 census[16];  // debug snapshot (see census())
   u64 stats[32];
@@ -120,6 +122,7 @@ struct Ctx {
   u64 timeout_ns;
   u64 census_ns;   // debug: take a state census this long after the kernel started (0 = never)
   u32 max_iters;
+  u32 blocking;    // 1: a warp waits in place for its query's pages instead of yielding
 };
 
 // launchers implemented in search_kernels.cu

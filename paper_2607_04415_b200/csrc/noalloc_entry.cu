@@ -123,9 +123,10 @@ extern "C" int gorio_search_resident_noalloc(const gorio_index_desc *d, const vo
   c.host_pages = (const u8 *)pages_dev;
   const u32 runq = 2 * kNaSlots, arrq = 1024, smallq = 256;
   u32 *qh = c.ctl->q_heads;
-  c.arr = Queue{(u32 *)cv.take<u64>(arrq), arrq - 1, qh + 0, qh + 1, (int *)(qh + 2)};
-  c.run = Queue{(u32 *)cv.take<u64>(runq), runq - 1, qh + 3, qh + 4, (int *)(qh + 5)};
-  c.want = Queue{(u32 *)cv.take<u64>(smallq), smallq - 1, qh + 6, qh + 7, (int *)(qh + 8)};
+  int *cnt = c.ctl->counts;
+  c.arr = Queue{(u32 *)cv.take<u64>(arrq), arrq - 1, qh + 0, qh + 1, cnt + 2};
+  c.run = Queue{(u32 *)cv.take<u64>(runq), runq - 1, qh + 3, qh + 4, cnt + 3};
+  c.want = Queue{(u32 *)cv.take<u64>(smallq), smallq - 1, qh + 6, qh + 7, cnt + 4};
   c.n_qslots = slots; c.nq = nq; c.K = K; c.L = L; c.W = W; c.WR = WR;
   c.hdr = cv.take<QHdr>(slots);
   c.list = cv.take<u64>((size_t)slots * L); c.cand = cv.take<u64>((size_t)slots * WR);
@@ -141,6 +142,7 @@ extern "C" int gorio_search_resident_noalloc(const gorio_index_desc *d, const vo
   c.timeout_ns = 60ull * 1000000000ull;
   c.census_ns = 0;
   c.max_iters = 64u * L + 1024u;
+  c.blocking = 0;
 
   // The array keeps the previous call's contents: reset everything that must start clean.
   const size_t ring_bytes = (size_t)((unsigned char *)(c.fdone + kNaRing) - (unsigned char *)dummy);

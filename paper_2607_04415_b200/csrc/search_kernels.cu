@@ -49,6 +49,11 @@ __device__ __forceinline__ u32 ld_sys_u32(const u32 *p) {
 __device__ __forceinline__ u64 ld_sys_u64(const u64 *p) {
   u64 v; asm volatile("ld.relaxed.sys.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory"); return v;
 }
+__device__ __forceinline__ uint4 ld_v4(const u32 *p) {
+  uint4 v;
+  asm volatile("ld.relaxed.gpu.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  return v;
+}
 __device__ __forceinline__ uint4 ld_sys_v4(const u32 *p) {
   uint4 v;
   asm volatile("ld.volatile.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
@@ -340,7 +345,7 @@ __device__ void consume_item(const Ctx &c, u32 qs, u32 j, u32 slot, u32 lane) {
 __device__ __forceinline__ void complete_items(const Ctx &c, u32 qs, u32 n) {
   __threadfence();
   u32 old = atomicSub(&c.hdr[qs].awaiting, n);
-  if (old == n) { q_push(c, c.run, qs, false); stat_add(c, S_RESUMES, 1); }
+  if (old == n) { if (!c.blocking) q_push(c, c.run, qs, false); stat_add(c, S_RESUMES, 1); }
   else if (old < n) raise(c, 8, 0x61, qs, old, n);
 }
 
@@ -942,6 +947,54 @@ __device__ bool recycle_slot(const Ctx &c, u32 qs, u32 lane) {
   return true;
 }
 
+__device__ void copy_page(const Ctx &c, u32 idx, u32 lane);
+__device__ bool warp_ticket(int *count, u32 *head, u32 &idx, u32 lane);
+
+// One unit of the work that keeps pages moving, in priority order: execute a copy the proxy
+// has admitted, consume a page the proxy has published (or a handed-off waiter chain), give
+// a waiting page a slot.  Returns 0 if there was nothing to do, 1 for a copy, 2 for an arrival.
+__device__ __noinline__ u32 service_step(const Ctx &c, u32 lane) {
+  u32 v;
+  if (warp_ticket(&c.ctl->counts[0], &c.cs->copy_head, v, lane)) {    // the outstanding window waits on these
+    copy_page(c, v, lane);
+    return 1;
+  }
+  if (warp_ticket(&c.ctl->counts[1], &c.cs->comp_head, v, lane)) {    // completion v: its page has arrived
+    const u64 e = __shfl_sync(0xffffffffu, ld_u64(c.ring_dev + (v & c.ring_mask)), 0);
+    consume_arrival(c, (u32)(e >> 8) & 0xFFFFFFu, lane);
+    return 2;
+  }
+  if (warp_pop(c, c.arr, v, lane)) {                                  // handed-off waiter chains
+    consume_arrival(c, v, lane);
+    return 2;
+  }
+  return 0;
+}
+__device__ void idle_step(const Ctx &c, u32 lane) {
+  // nothing else to do: see whether a page waiting for a slot can be given one
+  if (lane == 0 && (int)ld_u32((const u32 *)c.want.count) > 0) {
+    LaneStats st = {0, 0, 0, 0, 0, 0};
+    serve_want(c, kNil, st);
+    stat_add(c, S_EVICT, st.evict); stat_add(c, S_POSTED, st.posted);
+  }
+  __syncwarp();
+}
+
+// Blocking mode (the demand-paging baseline the paper compares against, Section 5.1: misses
+// "issue remote reads and wait for page readiness"): the warp keeps its query and waits in
+// place until the batch it issued is complete.  It still moves pages while it waits -- someone
+// has to -- but it never picks up another query, so at most one query per warp is in flight.
+__device__ __noinline__ bool wait_in_place(const Ctx &c, u32 qs, u32 lane) {
+  const u64 t0 = globaltimer();
+  for (u32 it = 0;; ++it) {
+    if (uld(&c.hdr[qs].awaiting) == 0u) { __threadfence(); return true; }
+    if (warp_stopped(c)) return false;
+    if (service_step(c, lane) == 0) { idle_step(c, lane); __nanosleep(200); }
+    u32 late = ((it & 255u) == 255u && globaltimer() - t0 > c.timeout_ns) ? 1u : 0u;
+    if (__shfl_sync(0xffffffffu, late, 0)) { if (lane == 0) raise(c, 5, 0xB5, qs); return false; }
+  }
+}
+
 template <bool PQ>
 __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut) {
   QHdr *h = c.hdr + qs;
@@ -962,7 +1015,7 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut) {
         if (lane == 0) st_u64(c.cand + (u64)qs * c.WR, mk_key(d, c.entry));
         __syncwarp();
       } else {
-        if (!issue_batch(c, qs, lane)) return;
+        if (!issue_batch(c, qs, lane) && !(c.blocking && wait_in_place(c, qs, lane))) return;
       }
     } else if (phase == PH_EVAL) {
       const u32 nf = merge_select_dispatch(c, qs, lane);
@@ -979,7 +1032,7 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut) {
         if (it > c.max_iters) raise(c, 6, 0xA1, qs, it);
       }
       __syncwarp();
-      if (!issue_batch(c, qs, lane)) return;
+      if (!issue_batch(c, qs, lane) && !(c.blocking && wait_in_place(c, qs, lane))) return;
     } else {  // PH_EXPAND complete
       const u32 nf = uld(&h->n_items);
       const u32 nn = collect_neighbors(c, qs, lane);
@@ -997,7 +1050,7 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut) {
       if (lane == 0) { st_u32(&h->n_items, nn); st_u32(&h->phase, PH_EVAL); }
       __syncwarp();
       if (!PQ && nn > 0) {
-        if (!issue_batch(c, qs, lane)) return;
+        if (!issue_batch(c, qs, lane) && !(c.blocking && wait_in_place(c, qs, lane))) return;
       }
     }
   }
@@ -1060,7 +1113,7 @@ __device__ void census(const Ctx &c, u32 lane) {
   for (int i = 0; i < 12; ++i) cnt[i] = __reduce_add_sync(0xffffffffu, cnt[i]);
   if (lane == 0) {
     for (int i = 0; i < 9; ++i) c.ctl->census[i] = cnt[i];
-    c.ctl->census[9] = (u32)*c.want.count; c.ctl->census[10] = (u32)c.cs->comp_count; c.ctl->census[11] = (u32)*c.run.count;
+    c.ctl->census[9] = (u32)*c.want.count; c.ctl->census[10] = (u32)c.ctl->counts[1]; c.ctl->census[11] = (u32)*c.run.count;
     c.ctl->census[12] = ld_u32(&c.ctl->done); c.ctl->census[13] = ld_u32(&c.ctl->ring_head);
   }
 }
@@ -1082,8 +1135,8 @@ __device__ void poller(const Ctx &c, u32 lane) {
     if (lane == 0) {
       const uint4 h = ld_sys_v4(c.host_ctl);
       pub = h.x; abort_req = h.y; adm = h.z;
-      if (adm != seen_adm) atomicAdd(&c.cs->copy_count, (int)(adm - seen_adm));
-      if (pub != seen_pub) atomicAdd(&c.cs->comp_count, (int)(pub - seen_pub));
+      if (adm != seen_adm) atomicAdd(&c.ctl->counts[0], (int)(adm - seen_adm));
+      if (pub != seen_pub) atomicAdd(&c.ctl->counts[1], (int)(pub - seen_pub));
       if (adm == seen_adm && pub == seen_pub) __nanosleep(100);
       seen_adm = adm; seen_pub = pub;
     }
@@ -1101,7 +1154,7 @@ __device__ __forceinline__ bool take_ticket(int *count, u32 *head, u32 &idx) {
   idx = atomicAdd(head, 1u);
   return true;
 }
-__device__ __forceinline__ bool warp_ticket(int *count, u32 *head, u32 &idx, u32 lane) {
+__device__ bool warp_ticket(int *count, u32 *head, u32 &idx, u32 lane) {
   u32 ok = 0, v = 0;
   if (lane == 0) ok = take_ticket(count, head, v) ? 1u : 0u;
   idx = __shfl_sync(0xffffffffu, v, 0);
@@ -1124,20 +1177,30 @@ __global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
   for (;;) {
     if (warp_stopped(c)) break;
     u32 v;
-    if (warp_ticket(&c.cs->copy_count, &c.cs->copy_head, v, lane)) {   // the outstanding window waits on these
-      copy_page(c, v, lane); idle = 0;
-      const u64 t = globaltimer(); t_cpy += t - tp; tp = t;
-      continue;
+    if (idle) {
+      // idle warps look at all five work counters with one 32-byte read (they sit together in
+      // the control block) and back off exponentially: thousands of warps polling five hot
+      // words would otherwise delay the very ticket atomics that hand out the work
+      u32 any = 0;
+      if (lane == 0) {
+        const uint4 a = ld_v4((const u32 *)&c.ctl->counts[0]);
+        const int w5 = (int)ld_u32((const u32 *)&c.ctl->counts[4]);
+        any = ((int)a.x > 0 || (int)a.y > 0 || (int)a.z > 0 || (int)a.w > 0 || w5 > 0) ? 1u : 0u;
+      }
+      if (!__shfl_sync(0xffffffffu, any, 0)) {
+        ++idle;
+        __nanosleep(idle < 7 ? (64u << idle) : 8000u);
+        u32 late = ((idle & 127u) == 0 && globaltimer() - t0 > c.timeout_ns) ? 1u : 0u;
+        if (__shfl_sync(0xffffffffu, late, 0)) { if (lane == 0) raise(c, 5, 0xB3); break; }
+        { const u64 t = globaltimer(); t_idle += t - tp; tp = t; }
+        continue;
+      }
     }
-    if (warp_ticket(&c.cs->comp_count, &c.cs->comp_head, v, lane)) {   // completion v: its page has arrived
-      const u64 e = __shfl_sync(0xffffffffu, ld_u64(c.ring_dev + (v & c.ring_mask)), 0);
-      consume_arrival(c, (u32)(e >> 8) & 0xFFFFFFu, lane); idle = 0;
-      const u64 t = globaltimer(); t_arr += t - tp; tp = t; ++n_arr;
-      continue;
-    }
-    if (warp_pop(c, c.arr, v, lane)) {             // handed-off waiter chains
-      consume_arrival(c, v, lane); idle = 0;
-      const u64 t = globaltimer(); t_arr += t - tp; tp = t; ++n_arr;
+    if (const u32 what = service_step(c, lane)) {
+      idle = 0;
+      const u64 t = globaltimer();
+      if (what == 1) t_cpy += t - tp; else { t_arr += t - tp; ++n_arr; }
+      tp = t;
       continue;
     }
     if (warp_pop(c, c.run, v, lane)) {
@@ -1145,16 +1208,8 @@ __global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
       const u64 t = globaltimer(); t_run += t - tp; tp = t; ++n_run;
       continue;
     }
-    // nothing to run: see whether a page waiting for a slot can be given one
-    if (lane == 0 && (int)ld_u32((const u32 *)c.want.count) > 0) {
-      LaneStats st = {0, 0, 0, 0, 0, 0};
-      serve_want(c, kNil, st);
-      stat_add(c, S_EVICT, st.evict); stat_add(c, S_POSTED, st.posted);
-    }
+    idle_step(c, lane);
     ++idle;
-    __nanosleep(idle < 16 ? 100 : 1000);
-    u32 late = ((idle & 127u) == 0 && globaltimer() - t0 > c.timeout_ns) ? 1u : 0u;
-    if (__shfl_sync(0xffffffffu, late, 0)) { if (lane == 0) raise(c, 5, 0xB3); break; }
     { const u64 t = globaltimer(); t_idle += t - tp; tp = t; }
   }
   if (lane == 0) {
@@ -1181,10 +1236,11 @@ __global__ void init_kernel(const Ctx c) {
     Ctl *ctl = c.ctl;
     ctl->stop = 0; ctl->status = 0; ctl->next_query = c.n_qslots; ctl->done = 0; ctl->ring_head = 0;
     for (int i = 0; i < 16; ++i) ctl->q_heads[i] = 0;
+    for (int i = 0; i < 8; ++i) ctl->counts[i] = 0;
     for (int i = 0; i < 8; ++i) ctl->dbg[i] = 0;
     *c.run.tail = c.n_qslots;
     *c.run.count = (int)c.n_qslots;
-    c.cs->copy_count = 0; c.cs->copy_head = 0; c.cs->comp_count = 0; c.cs->comp_head = 0;
+    ctl->counts[0] = 0; ctl->counts[1] = 0; c.cs->copy_head = 0; c.cs->comp_head = 0;
   }
 }
 

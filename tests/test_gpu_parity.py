@@ -105,6 +105,8 @@ def test_cold_cache_with_room_for_every_page_fetches_each_page_once(gorio, cfg1)
     dict(capacity=1000, max_outstanding=4), dict(capacity=1000, max_outstanding=1024),
     dict(capacity=2500, tuning=dict(warps_per_block=4)), dict(capacity=2500, tuning=dict(max_inflight=48)),
     dict(capacity=2500, tuning=dict(warps_per_block=8, blocks_per_sm=2)),
+    dict(capacity=1000, remote_latency_ns=20000, tuning=dict(blocking=1)),
+    dict(capacity=1000, tuning=dict(stash_entries=1)), dict(capacity=1000, tuning=dict(stash_entries=64)),
 ], ids=lambda c: "-".join(f"{k}={v}" for k, v in c.items() if k != "tuning") + ("-tuned" if "tuning" in c else ""))
 def test_results_do_not_depend_on_cache_proxy_or_geometry(gorio, cfg1, cfg):
     """The proxy never touches search state, so outputs must be identical under any cache
@@ -336,3 +338,21 @@ def test_config5_scaled_fp32_tolerance(gorio):
     ref = OracleIndex.from_workload(w).search(w.queries, w.K, w.L, w.W, threads=8)
     got = _gpu_search(gorio, w, w.cache_pages, remote_latency_ns=20000, max_outstanding=256)
     _fp32_parity(w, got, ref)
+
+
+def test_config5_full_size_sampled_fp32_tolerance(gorio):
+    """10,000,000 x 96 fp32 nodes, 6 per page (1,666,667 pages, 6.8 GB pinned), 10,000 queries,
+    K=10 L=128 W=4, 10 % cache, 20 us; the oracle checks every 50th query."""
+    w = make_config(5)
+    assert w.N == 10_000_000 and w.n_pages == 1_666_667 and w.node_bytes == 644
+    sample = np.arange(0, w.nq, 50)
+    ref = OracleIndex.from_workload(w).search(w.queries[sample], w.K, w.L, w.W, threads=8)
+    got = _gpu_search(gorio, w, w.cache_pages, remote_latency_ns=20000, max_outstanding=256, timeout_ms=120000)
+    _fp32_parity(w, got, ref, rows=sample)
+    assert got["stats"]["queries_done"] == w.nq and got["stats"]["max_outstanding_seen"] <= 256
+    # properties at full size: reported distances recomputable in double within fp32 rounding
+    for r in range(0, w.nq, 211):
+        ids = got["ids"][r]
+        dd = ((w.data[ids].astype(np.float64) - w.queries[r].astype(np.float64)) ** 2).sum(1)
+        np.testing.assert_allclose(got["dists"][r], dd, rtol=2e-6)
+        assert (np.diff(dd) >= -1e-5 * dd[1:]).all()
