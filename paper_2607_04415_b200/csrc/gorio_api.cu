@@ -498,6 +498,8 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   c.timeout_ns = (u64)ix->cfg.timeout_ms * 1000000ull;
   c.max_iters = 64u * L + 1024u;
   c.blocking = ix->tune.blocking ? 1u : 0u;
+  c.vec128 = (ix->vec_bytes % 16 == 0 && ix->vec_bytes <= 384 && ((uintptr_t)queries_dev & 15) == 0 &&
+              !std::getenv("GORIO_NO_VEC128")) ? 1u : 0u;
   { const char *e = std::getenv("GORIO_CENSUS_MS"); c.census_ns = e ? (u64)std::atof(e) * 1000000ull : 0; }
 
   // launch geometry: leave room on every SM for the proxy's copy kernels

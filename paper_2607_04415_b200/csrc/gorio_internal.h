@@ -122,6 +122,7 @@ struct Ctx {
   u64 timeout_ns;
   u64 census_ns;   // debug: take a state census this long after the kernel started (0 = never)
   u32 max_iters;
+  u32 vec128;      // 1: vectors are whole 16-byte chunks (<= 24) and query rows are 16-byte aligned
   u32 blocking;    // 1: a warp waits in place for its query's pages instead of yielding
 };
 

@@ -143,6 +143,8 @@ extern "C" int gorio_search_resident_noalloc(const gorio_index_desc *d, const vo
   c.census_ns = 0;
   c.max_iters = 64u * L + 1024u;
   c.blocking = 0;
+  c.vec128 = (c.vec_bytes % 16 == 0 && c.vec_bytes <= 384 && ((uintptr_t)queries_dev & 15) == 0 &&
+              ((uintptr_t)pages_dev & 15) == 0) ? 1u : 0u;
 
   // The array keeps the previous call's contents: reset everything that must start clean.
   const size_t ring_bytes = (size_t)((unsigned char *)(c.fdone + kNaRing) - (unsigned char *)dummy);
