@@ -985,6 +985,18 @@ __device__ __forceinline__ u32 warp_adc(const Ctx &c, const u32 *lut, u32 v, u32
   for (u32 m = lane; m < c.pq_m; m += 32) acc += lut[(m << 8) + __ldg(code + m)];
   return __reduce_add_sync(0xffffffffu, acc);
 }
+// One node per lane: the lane reads the node's code (pq_m bytes, 4 at a time) and sums pq_m
+// independent table entries from shared memory -- no cross-lane reduction, 32 nodes per pass.
+__device__ __forceinline__ u32 lane_adc(const Ctx &c, const u32 *lut, u32 v) {
+  const u32 *code = (const u32 *)(c.pq_codes + (u64)v * c.pq_m);
+  u32 acc = 0;
+  for (u32 w = 0; w < (c.pq_m >> 2); ++w) {
+    const u32 cw = __ldg(code + w);
+    acc += lut[((4u * w + 0u) << 8) + (cw & 255u)] + lut[((4u * w + 1u) << 8) + ((cw >> 8) & 255u)] +
+           lut[((4u * w + 2u) << 8) + ((cw >> 16) & 255u)] + lut[((4u * w + 3u) << 8) + (cw >> 24)];
+  }
+  return acc;
+}
 
 // ------------------------------------------------------------------------------------------
 // query life cycle
@@ -1085,8 +1097,10 @@ __device__ __noinline__ bool wait_in_place(const Ctx &c, u32 qs, u32 lane) {
   }
 }
 
+// lut_qid: the query whose table currently sits in this warp's shared memory (kept across calls,
+// so a query that runs several phases in a row on one warp builds its table once).
 template <bool PQ>
-__device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut) {
+__device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut, u32 &lut_qid) {
   QHdr *h = c.hdr + qs;
   for (u32 guard = 0; guard < 4u * c.max_iters + 64u; ++guard) {
     if (warp_stopped(c)) return;
@@ -1100,7 +1114,7 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut) {
       }
       __syncwarp();
       if (PQ) {
-        build_lut(c, qid, lut, lane);
+        if (lut_qid != qid) { build_lut(c, qid, lut, lane); lut_qid = qid; }
         u32 d = warp_adc(c, lut, c.entry, lane);
         if (lane == 0) st_u64(c.cand + (u64)qs * c.WR, mk_key(d, c.entry));
         __syncwarp();
@@ -1129,13 +1143,16 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut) {
       if (PQ) {
         pool_merge_dispatch(c, qs, nf, false, lane);
         const u32 qid = uld(&h->qid);
-        build_lut(c, qid, lut, lane);
+        if (lut_qid != qid) { build_lut(c, qid, lut, lane); lut_qid = qid; }
         const u32 *items = c.items + (u64)qs * c.WR;
-        for (u32 i = 0; i < nn; ++i) {
-          const u32 v = ld_u32(items + i);
-          u32 d = warp_adc(c, lut, v, lane);
-          if (lane == 0) st_u64(c.cand + (u64)qs * c.WR + i, mk_key(d, v));
+        for (u32 base = 0; base < nn; base += 32) {
+          const u32 i = base + lane;
+          if (i < nn) {
+            const u32 v = ld_u32(items + i);
+            st_u64(c.cand + (u64)qs * c.WR + i, mk_key(lane_adc(c, lut, v), v));
+          }
         }
+        __syncwarp();
       }
       if (lane == 0) { st_u32(&h->n_items, nn); st_u32(&h->phase, PH_EVAL); }
       __syncwarp();
@@ -1263,6 +1280,7 @@ __global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
   u32 idle = 0;
   // where the worker warps' time goes (ns, summed over warps): arrivals, query phases, idle
   u64 t_arr = 0, t_run = 0, t_idle = 0, t_cpy = 0, n_arr = 0, n_run = 0;
+  u32 lut_qid = kInvalidId;
   u64 tp = t0;
   for (;;) {
     if (warp_stopped(c)) break;
@@ -1294,7 +1312,7 @@ __global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
       continue;
     }
     if (warp_pop(c, c.run, v, lane)) {
-      run_query<PQ>(c, v, lane, lut); idle = 0;
+      run_query<PQ>(c, v, lane, lut, lut_qid); idle = 0;
       const u64 t = globaltimer(); t_run += t - tp; tp = t; ++n_run;
       continue;
     }
