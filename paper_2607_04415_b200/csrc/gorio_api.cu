@@ -502,7 +502,7 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
               !std::getenv("GORIO_NO_VEC128")) ? 1u : 0u;
   { const char *e = std::getenv("GORIO_CENSUS_MS"); c.census_ns = e ? (u64)std::atof(e) * 1000000ull : 0; }
 
-  // launch geometry: leave room on every SM for the proxy's copy kernels
+  // launch geometry: one block per SM by default
   const bool pq = d.pq_m != 0;
   // default warps per SM: 24 when pages will be missed (arrivals are served by whoever is free);
   // with every page resident one warp carries one query at a time, so no more than there are

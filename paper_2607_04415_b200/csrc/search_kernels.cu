@@ -1268,8 +1268,7 @@ __device__ bool warp_ticket(int *count, u32 *head, u32 &idx, u32 lane) {
   return __shfl_sync(0xffffffffu, ok, 0) != 0u;
 }
 
-// Register budget: at most 80 per thread, so that 20 resident warps leave register file and
-// thread slots on every SM for the proxy's copy kernels, which must run concurrently.
+// Register budget: at most 80 per thread, so that 24 warps (61,440 registers) fit on an SM.
 template <bool PQ>
 __global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
   extern __shared__ u32 smem_lut[];
