@@ -109,6 +109,9 @@ typedef struct {
  *                    table that keeps a scored node's neighbour list so that expanding it later
  *                    needs no page; 0 = default 1024, 1 = off, else a power of two >= 64.
  *                    It never changes results, only how many pages are waited for.
+ *   request_backlog  most requests posted to the proxy and not yet arrived; 0 = default
+ *                    4 * max_outstanding.  More than the proxy can have in service only queues
+ *                    in the ring while occupying cache slots that could hold resident pages.
  *   blocking         1 = ablation: a warp that misses keeps its query and waits in place for
  *                    the pages (the demand-paging baseline of Section 5.1) instead of parking
  *                    the query and taking another; results are identical, only slower.
@@ -120,6 +123,8 @@ typedef struct {
   uint32_t blocks_per_sm;
   uint32_t stash_entries;
   uint32_t blocking;
+  uint32_t request_backlog;
+  uint32_t reserved;
 } gorio_tuning;
 
 /*

@@ -57,7 +57,7 @@ struct gorio_index {
 
   // query state
   gorio_tuning tune{};
-  u32 qs_slots = 0, qs_L = 0, qs_W = 0, qs_WR = 0, qs_K = 0, qs_seen = 0, qs_pset = 0, qs_stash = 0;
+  u32 qs_slots = 0, qs_L = 0, qs_W = 0, qs_WR = 0, qs_K = 0, qs_seen = 0, qs_pset = 0, qs_stash = 0, qs_nslots = 0;
   void *qs_block = nullptr;
   Ctx ctx{};
   Ctl *ctl = nullptr;
@@ -255,7 +255,6 @@ int setup_cache(gorio_index *ix) {
   ix->n_slots = cap >= ix->n_pages ? ix->n_pages : (u32)cap;
   ix->ring_cap = next_pow2(2ull * ix->n_slots < 1024 ? 1024 : 2ull * ix->n_slots);
   ix->want_cap = next_pow2(ix->n_pages < 64 ? 64 : ix->n_pages);
-  free_qstate(ix);               // the arrival queue is sized from the slot count
   CK(cudaMalloc(&ix->slot_data, (size_t)ix->n_slots * kPageBytes));
   CK(cudaMalloc(&ix->ptab, (size_t)ix->n_pages * 8));
   CK(cudaMalloc(&ix->smeta, (size_t)ix->n_slots * 8));
@@ -288,7 +287,8 @@ int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W) {
   const u32 seen_cap = ix->tune.visited_capacity ? ix->tune.visited_capacity : 32768u;
   const u32 pset_cap = ix->desc.pq_m ? 4096u : seen_cap;
   if (ix->qs_block && ix->qs_slots >= slots && ix->qs_L == L && ix->qs_W == W && ix->qs_K == K &&
-      ix->qs_seen == seen_cap && ix->qs_pset == pset_cap && ix->qs_stash == (ix->tune.stash_entries + 1u)) {
+      ix->qs_seen == seen_cap && ix->qs_pset == pset_cap && ix->qs_stash == (ix->tune.stash_entries + 1u) &&
+      ix->qs_nslots == ix->n_slots) {      // (the arrival queue and the stash default depend on the slot count)
     ix->ctx.n_qslots = slots;
     return GORIO_OK;
   }
@@ -326,7 +326,7 @@ int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W) {
   c.stash_tag = (u32 *)(b + o_stag); c.stash = (u32 *)(b + o_stash); c.stash_cap = stash_cap;
   c.seen_cap = seen_cap; c.pset_cap = pset_cap; c.n_qslots = slots;
   ix->qs_slots = slots; ix->qs_L = L; ix->qs_W = W; ix->qs_WR = WR; ix->qs_K = K;
-  ix->qs_seen = seen_cap; ix->qs_pset = pset_cap; ix->qs_stash = ix->tune.stash_entries + 1u;
+  ix->qs_seen = seen_cap; ix->qs_pset = pset_cap; ix->qs_stash = ix->tune.stash_entries + 1u; ix->qs_nslots = ix->n_slots;
   return GORIO_OK;
 }
 
@@ -498,16 +498,18 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   c.timeout_ns = (u64)ix->cfg.timeout_ms * 1000000ull;
   c.max_iters = 64u * L + 1024u;
   c.blocking = ix->tune.blocking ? 1u : 0u;
-  c.vec128 = (ix->vec_bytes % 16 == 0 && ix->vec_bytes <= 384 && ((uintptr_t)queries_dev & 15) == 0 &&
-              !std::getenv("GORIO_NO_VEC128")) ? 1u : 0u;
+  c.idle_ns = 8000u;
+  c.max_in_flight = ix->tune.request_backlog ? ix->tune.request_backlog : 4u * ix->cfg.max_outstanding;
+  if (c.max_in_flight < ix->cfg.max_outstanding) c.max_in_flight = ix->cfg.max_outstanding;
+  c.vec128 = (ix->vec_bytes % 16 == 0 && ix->vec_bytes <= 384 && ((uintptr_t)queries_dev & 15) == 0) ? 1u : 0u;
   { const char *e = std::getenv("GORIO_CENSUS_MS"); c.census_ns = e ? (u64)std::atof(e) * 1000000ull : 0; }
 
   // launch geometry: one block per SM by default
   const bool pq = d.pq_m != 0;
-  // default warps per SM: 24 when pages will be missed (arrivals are served by whoever is free);
+  // default warps per SM: 16 when pages will be missed (more warps lengthen every copy and arrival);
   // with every page resident one warp carries one query at a time, so no more than there are
   // queries per SM (fewer idle warps polling the queues), within 8..24
-  u32 auto_warps = 24u;
+  u32 auto_warps = 16u;
   if (ix->n_slots >= ix->n_pages) {
     auto_warps = (nq + (u32)ix->n_sms - 1) / (u32)ix->n_sms;
     auto_warps = auto_warps < 8u ? 8u : (auto_warps > 24u ? 24u : auto_warps);

@@ -51,6 +51,7 @@ struct CacheShared {
   u32 bump;
   u32 copy_head;   // next admitted request to copy
   u32 comp_head;   // next published completion to consume
+  int in_flight;   // requests posted whose arrival has not been picked up yet
 };
 
 // Device-resident control block.
@@ -122,6 +123,8 @@ struct Ctx {
   u64 timeout_ns;
   u64 census_ns;   // debug: take a state census this long after the kernel started (0 = never)
   u32 max_iters;
+  u32 idle_ns;       // longest sleep of an idle warp between looks at the work counters
+  u32 max_in_flight; // cap on posted-but-not-arrived requests
   u32 vec128;      // 1: vectors are whole 16-byte chunks (<= 24) and query rows are 16-byte aligned
   u32 blocking;    // 1: a warp waits in place for its query's pages instead of yielding
 };

@@ -174,6 +174,7 @@ struct LaneStats { u32 hit, missed, joins, evict, retry, posted; };
 // target cache slot, publish through a ready flag -- here the lap tag inside the word.)
 __device__ __forceinline__ void post_request(const Ctx &c, u32 page, u32 slot) {
   const u32 idx = atomicAdd(&c.ctl->ring_head, 1u);
+  atomicAdd(&c.cs->in_flight, 1);
   const u32 lap = ((idx >> c.ring_shift) % 255u) + 1u;
   const u64 e = ((u64)page << 32) | ((u64)slot << 8) | lap;
   st_u64(c.ring_dev + (idx & c.ring_mask), e);   // device copy: what copy and arrival tickets refer to
@@ -189,7 +190,7 @@ __device__ u32 alloc_slot(const Ctx &c, u32 hint, LaneStats &st) {
     u32 b = atomicAdd(&c.cs->bump, 1u);
     if (b < c.n_slots) return b;
   }
-  const int sweep = hint != kNil ? 2 : 48;
+  const int sweep = hint != kNil ? 6 : 48;
   for (int step = 0; step <= sweep; ++step) {
     const bool use_hint = step == sweep;
     if (use_hint && hint == kNil) break;
@@ -226,8 +227,14 @@ __device__ void assign_and_post(const Ctx &c, u32 page, u32 slot, LaneStats &st)
 }
 
 // Serve one page from the want queue if a slot can be had (one lane).
+// Requests posted and not yet arrived are kept near a small multiple of the proxy's window:
+// anything more would only queue in the ring while holding a slot that could keep a resident
+// page instead (with the whole cache in flight it is a buffer pool, not a cache).
+__device__ __forceinline__ bool may_post(const Ctx &c) { return (int)ld_u32((const u32 *)&c.cs->in_flight) < (int)c.max_in_flight; }
+
 __device__ void serve_want(const Ctx &c, u32 hint, LaneStats &st) {
   u32 page;
+  if (!may_post(c)) return;
   if (!q_pop(c, c.want, page)) return;
   const u32 slot = alloc_slot(c, hint, st);
   if (slot == kNil) { q_push(c, c.want, page); return; }
@@ -249,7 +256,7 @@ __device__ u32 page_lookup(const Ctx &c, u32 page, u32 g, u32 &slot, u32 &gen, L
     if (s == P_ABSENT) {
       if (atomicCAS((unsigned long long *)pw, w, mk_pw(P_WANTED, 0, g)) != w) continue;
       st.missed++;
-      const u32 sl = alloc_slot(c, kNil, st);          // first requester: find the page a slot
+      const u32 sl = may_post(c) ? alloc_slot(c, kNil, st) : kNil;   // first requester: find the page a slot
       if (sl != kNil) assign_and_post(c, page, sl, st);
       else q_push(c, c.want, page);
       return LK_WAIT;
@@ -612,6 +619,7 @@ __device__ void consume_arrival(const Ctx &c, u32 v, u32 lane) {
   if (__shfl_sync(0xffffffffu, bad, 0)) return;
   if (lane == 0) {
     st_u32(c.parts + slot, 1u);
+    atomicSub(&c.cs->in_flight, 1);
     st_u64(c.smeta + slot, m | 1ull);                      // a fresh page gets its second chance
     const u64 old = atomicExch((unsigned long long *)(c.ptab + page), mk_pw(P_ARRIVED, slot, gen));
     if (pw_state(old) != P_FILLING || pw_slot(old) != slot) { raise(c, 8, 0x72, slot, page, (u32)(old >> 32)); bad = 1; }
@@ -1296,7 +1304,7 @@ __global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
       }
       if (!__shfl_sync(0xffffffffu, any, 0)) {
         ++idle;
-        __nanosleep(idle < 7 ? (64u << idle) : 8000u);
+        __nanosleep(idle < 7 ? (64u << idle) : c.idle_ns);
         u32 late = ((idle & 127u) == 0 && globaltimer() - t0 > c.timeout_ns) ? 1u : 0u;
         if (__shfl_sync(0xffffffffu, late, 0)) { if (lane == 0) raise(c, 5, 0xB3); break; }
         { const u64 t = globaltimer(); t_idle += t - tp; tp = t; }
@@ -1347,7 +1355,7 @@ __global__ void init_kernel(const Ctx c) {
     for (int i = 0; i < 8; ++i) ctl->dbg[i] = 0;
     *c.run.tail = c.n_qslots;
     *c.run.count = (int)c.n_qslots;
-    ctl->counts[0] = 0; ctl->counts[1] = 0; c.cs->copy_head = 0; c.cs->comp_head = 0;
+    ctl->counts[0] = 0; ctl->counts[1] = 0; c.cs->copy_head = 0; c.cs->comp_head = 0; c.cs->in_flight = 0;
   }
 }
 

@@ -106,6 +106,7 @@ def test_cold_cache_with_room_for_every_page_fetches_each_page_once(gorio, cfg1)
     dict(capacity=2500, tuning=dict(warps_per_block=4)), dict(capacity=2500, tuning=dict(max_inflight=48)),
     dict(capacity=2500, tuning=dict(warps_per_block=8, blocks_per_sm=2)),
     dict(capacity=1000, remote_latency_ns=20000, tuning=dict(blocking=1)),
+    dict(capacity=1000, tuning=dict(request_backlog=100000)), dict(capacity=1000, max_outstanding=8, tuning=dict(request_backlog=8)),
     dict(capacity=1000, tuning=dict(stash_entries=1)), dict(capacity=1000, tuning=dict(stash_entries=64)),
 ], ids=lambda c: "-".join(f"{k}={v}" for k, v in c.items() if k != "tuning") + ("-tuned" if "tuning" in c else ""))
 def test_results_do_not_depend_on_cache_proxy_or_geometry(gorio, cfg1, cfg):
