@@ -116,6 +116,9 @@ def main():
     ap.add_argument("--blocking", action="store_true", help="ablation: warps wait in place on a miss")
     ap.add_argument("--latency-us", type=float, default=None)
     ap.add_argument("--max-outstanding", type=int, default=None)
+    ap.add_argument("--sweep", default=None,
+                    help="comma list of latency_us:max_outstanding points; prints one short JSON line per point "
+                         "(characterisation runs, not the benchmark line)")
     ap.add_argument("--L", type=int, default=None)
     ap.add_argument("--W", type=int, default=None)
     args = ap.parse_args()
@@ -213,6 +216,27 @@ def main():
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t), out, ix.stats()
 
+    if args.sweep:
+        for point in args.sweep.split(","):
+            lat_us, mo = point.split(":")
+            lat_ns, max_out = int(float(lat_us) * 1000), int(mo)
+            ts, sts = [], []
+            for i in range(1 + max(1, args.steps)):
+                t, _, st_i = one_step()
+                if i:
+                    ts.append(t); sts.append(st_i)
+            ms_p = statistics.mean(ts)
+            f_p = statistics.mean(x["pages_fetched"] for x in sts)
+            terms_p = {"host_link": 4096 * f_p / (h2d * 1e9), "outstanding_window": f_p * lat_ns * 1e-9 / max_out}
+            bound_p = max(terms_p, key=terms_p.get)
+            if rank == 0:
+                print(json.dumps({"latency_us": float(lat_us), "max_outstanding": max_out, "qps": world * w.nq / (ms_p * 1e-3),
+                                  "ms_per_step": ms_p, "pages_fetched": f_p, "fetch_rate_M_per_s": f_p / ms_p / 1e3,
+                                  "bound": bound_p, "frac": terms_p[bound_p] / (ms_p * 1e-3),
+                                  "service_us": statistics.mean(x["proxy_service_ns"] / max(1, x["pages_fetched"]) for x in sts) / 1e3,
+                                  "blocking": bool(args.blocking)}))
+        ix.close()
+        return
     for _ in range(max(3, args.warmup)):
         one_step()
     sampler = ClockSampler(local); sampler.start()

@@ -110,7 +110,7 @@ typedef struct {
  *                    needs no page; 0 = default 1024, 1 = off, else a power of two >= 64.
  *                    It never changes results, only how many pages are waited for.
  *   request_backlog  most requests posted to the proxy and not yet arrived; 0 = default
- *                    4 * max_outstanding.  More than the proxy can have in service only queues
+ *                    min(4 * max_outstanding, 1024), never below max_outstanding.  More than the proxy can have in service only queues
  *                    in the ring while occupying cache slots that could hold resident pages.
  *   blocking         1 = ablation: a warp that misses keeps its query and waits in place for
  *                    the pages (the demand-paging baseline of Section 5.1) instead of parking

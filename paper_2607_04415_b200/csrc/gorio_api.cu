@@ -499,7 +499,10 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   c.max_iters = 64u * L + 1024u;
   c.blocking = ix->tune.blocking ? 1u : 0u;
   c.idle_ns = 8000u;
-  c.max_in_flight = ix->tune.request_backlog ? ix->tune.request_backlog : 4u * ix->cfg.max_outstanding;
+  // default backlog: 4 x the proxy's window, but no more than 1024 (about what keeps the host
+  // link busy) unless the window itself is larger
+  c.max_in_flight = ix->tune.request_backlog ? ix->tune.request_backlog
+                    : (4u * ix->cfg.max_outstanding < 1024u ? 4u * ix->cfg.max_outstanding : 1024u);
   if (c.max_in_flight < ix->cfg.max_outstanding) c.max_in_flight = ix->cfg.max_outstanding;
   c.vec128 = (ix->vec_bytes % 16 == 0 && ix->vec_bytes <= 384 && ((uintptr_t)queries_dev & 15) == 0) ? 1u : 0u;
   { const char *e = std::getenv("GORIO_CENSUS_MS"); c.census_ns = e ? (u64)std::atof(e) * 1000000ull : 0; }
