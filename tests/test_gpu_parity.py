@@ -357,3 +357,58 @@ def test_config5_full_size_sampled_fp32_tolerance(gorio):
         dd = ((w.data[ids].astype(np.float64) - w.queries[r].astype(np.float64)) ** 2).sum(1)
         np.testing.assert_allclose(got["dists"][r], dd, rtol=2e-6)
         assert (np.diff(dd) >= -1e-5 * dd[1:]).all()
+
+
+# ------------------------------------------------------------------ scoring paths off the standard shapes
+@pytest.mark.parametrize("kind,d,R", [
+    ("u8", 20, 12),      # 20-byte vectors: not whole 16-byte chunks -> 4-byte-per-lane path
+    ("u8", 256, 24),     # 16 chunks: two chunks per lane in the 128-bit path
+    ("u8", 512, 8),      # longer than the 128-bit path handles -> one-at-a-time path
+    ("f32", 36, 16),     # 144-byte vectors: 9 chunks
+    ("f32", 200, 20),    # 800-byte vectors -> one-at-a-time path
+])
+def test_other_dimensions_match_oracle(gorio, kind, d, R):
+    from workloads import node_bytes as nbytes
+    nb = nbytes(d, np.uint8 if kind == "u8" else np.float32, R)
+    npp = max(1, 4096 // nb)
+    w = make_workload("odd", kind, 6000, 6, 300, d, R - 4, 4, npp, clustered_knn=True, cross_only=False,
+                      K=10, L=48, W=3)
+    ref = OracleIndex.from_workload(w).search(w.queries, w.K, w.L, w.W, threads=4)
+    got = _gpu_search(gorio, w, max(16, w.n_pages // 5), remote_latency_ns=2000)
+    if kind == "u8":
+        _assert_exact(got, ref)
+    else:
+        _fp32_parity(w, got, ref)
+
+
+def test_queries_not_16_byte_aligned_take_the_narrow_path(gorio, cfg1):
+    w, ref = cfg1
+    ix = gorio.Index.from_workload(w)
+    try:
+        ix.cache_config(1500)
+        buf = torch.zeros(4 + 200 * w.d, dtype=torch.uint8, device="cuda")
+        q = buf[4:].view(200, w.d)                       # data pointer is 4 bytes past a 16-byte boundary
+        q.copy_(torch.as_tensor(w.queries[:200]))
+        assert q.data_ptr() % 16 == 4 and q.is_contiguous()
+        out = ix.search(q, w.K, w.L, w.W)
+        assert (_u32(out["ids"]) == ref["ids"][:200]).all() and (_u32(out["dists"]) == ref["dists"][:200]).all()
+        assert (_u32(out["counters"]) == ref["counters"][:200]).all()
+    finally:
+        ix.close()
+
+
+def test_second_search_reuses_the_warm_cache(gorio, cfg1):
+    w, ref = cfg1
+    ix = gorio.Index.from_workload(w)
+    try:
+        ix.cache_config(w.n_pages, preload=False)         # room for everything, cold
+        q = torch.as_tensor(w.queries).cuda()
+        a = ix.search(q, w.K, w.L, w.W)
+        f1 = ix.stats()["pages_fetched"]
+        b = ix.search(q, w.K, w.L, w.W)                   # same index, no cache_config in between
+        f2 = ix.stats()["pages_fetched"] - f1
+        for out in (a, b):
+            assert (_u32(out["ids"]) == ref["ids"]).all() and (_u32(out["counters"]) == ref["counters"]).all()
+        assert f1 == int(ref["page_union"].sum()) and f2 == 0
+    finally:
+        ix.close()
