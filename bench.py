@@ -28,6 +28,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 METRIC = "QPS @ recall@10, 1M x 128 uint8, 20% cache, 20us miss"
+# dram__bytes_read.sum + dram__bytes_write.sum of one search_kernel launch on the default workload
+# (config 3, 10,000 queries, cold 20 % cache), mean of 8 launches of a single-pass ncu capture of this
+# very command; see profiles/search_kernel_cfg3_launch_list.md.  Reported only for that workload.
+NCU_DRAM_BYTES_PER_LAUNCH_CFG3 = 20.18e9 + 28.23e9
 PAPER_CONTEXT = ("paper (L40S + ConnectX-6 NVMe-oF, SIFT1M): G-ABaM 5650 QPS = 4.89x over blocking BaM, "
                  "G-Gust 1.31x over GustANN; context only, other hardware and transport")
 
@@ -285,6 +289,9 @@ def main():
     else:
         ach, peak, unit = fetched / (ms * 1e-3) / 1e6, max_out / max(lat_ns * 1e-9, 1e-12) / 1e6, "Mfetch/s"
 
+    default_workload = (args.config == 3 and args.scale == 1.0 and args.nq is None and not args.preload and
+                        not args.blocking and args.cache_frac == 0.20 and args.latency_us is None and
+                        not args.max_outstanding and not args.L and not args.W)
     ids = out["ids"].cpu().numpy().view(np.uint32)
     recall = recall_at_k(ids, w.gt)
     line = {
@@ -304,7 +311,7 @@ def main():
                 "d2h_bytes_per_step": int(sum(v.numel() * 4 for v in outs_pin.values()))},
         "gpu_launches": int(launches),
         "roofline": {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": t_roof / (ms * 1e-3),
-                     "traffic": None, "peak_kind": f"hbm {pk_kind}; host link measured in this run ({h2d:.1f} GB/s)",
+                     "traffic": (NCU_DRAM_BYTES_PER_LAUNCH_CFG3 if default_workload else None), "peak_kind": f"hbm {pk_kind}; host link measured in this run ({h2d:.1f} GB/s)",
                      "terms_ms": {k: 1e3 * v for k, v in terms.items()},
                      "pages_fetched": fetched, "algorithmic_hbm_bytes": b_hbm,
                      "hbm_achieved_gbs": b_hbm / (ms * 1e-3) / 1e9, "hbm_peak_gbs": pk["hbm_gbs"]},
