@@ -73,7 +73,6 @@ struct gorio_index {
   std::condition_variable cv;
   std::atomic<int> px_state{PX_IDLE};
   std::atomic<int> px_stop{0};
-  std::atomic<int> px_active{0};
   std::atomic<int> px_error{0};
   cudaStream_t own_stream = nullptr;
   cudaEvent_t done_ev = nullptr;
@@ -188,7 +187,7 @@ void proxy_service(gorio_index *ix) {
       while (!inflight.empty()) {
         const InService &r = inflight.front();
         if (now - r.admitted < latency) break;
-        if (fdone[r.idx & ring_mask] != ((r.idx >> ring_shift) % 255u) + 1u) { ++ack_wait_iters; break; }
+        if ((fdone[r.idx & ring_mask] & 0xFFu) != ((r.idx >> ring_shift) % 255u) + 1u) { ++ack_wait_iters; break; }
         service_ns += (u64)std::chrono::duration_cast<std::chrono::nanoseconds>(now - r.admitted).count();
         ++ct; ++published;
         inflight.pop_front();
@@ -220,12 +219,10 @@ void proxy_main(gorio_index *ix) {
       ix->cv.wait(lk, [&] { return ix->px_state.load() != PX_IDLE; });
     }
     if (ix->px_state.load() == PX_EXIT) return;
-    ix->px_active.store(1, std::memory_order_release);
     proxy_service(ix);
     {
       std::lock_guard<std::mutex> lk(ix->mu);
       if (ix->px_state.load() != PX_EXIT) ix->px_state.store(PX_IDLE);
-      ix->px_active.store(0, std::memory_order_release);
     }
     ix->cv.notify_all();
   }

@@ -31,23 +31,11 @@ __device__ __forceinline__ u32 ld_u32(const u32 *p) {
 __device__ __forceinline__ u64 ld_u64(const u64 *p) {
   u64 v; asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory"); return v;
 }
-__device__ __forceinline__ u16 ld_u16(const u16 *p) {
-  u16 v; asm volatile("ld.relaxed.gpu.global.u16 %0, [%1];" : "=h"(v) : "l"(p) : "memory"); return v;
-}
 __device__ __forceinline__ void st_u32(u32 *p, u32 v) {
   asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void st_u64(u64 *p, u64 v) {
   asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-__device__ __forceinline__ void st_u16(u16 *p, u16 v) {
-  asm volatile("st.relaxed.gpu.global.u16 [%0], %1;" ::"l"(p), "h"(v) : "memory");
-}
-__device__ __forceinline__ u32 ld_sys_u32(const u32 *p) {
-  u32 v; asm volatile("ld.relaxed.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory"); return v;
-}
-__device__ __forceinline__ u64 ld_sys_u64(const u64 *p) {
-  u64 v; asm volatile("ld.relaxed.sys.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory"); return v;
 }
 __device__ __forceinline__ uint4 ld_v4(const u32 *p) {
   uint4 v;
@@ -65,7 +53,6 @@ __device__ __forceinline__ void st_sys_u32(u32 *p, u32 v) {
 __device__ __forceinline__ void st_sys_u64(u64 *p, u64 v) {
   asm volatile("st.relaxed.sys.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
-__device__ __forceinline__ void fence_sc() { asm volatile("fence.sc.gpu;" ::: "memory"); }
 __device__ __forceinline__ u64 globaltimer() {
   u64 t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t;
 }
@@ -82,7 +69,6 @@ __device__ __noinline__ void raise(const Ctx &c, u32 status, u32 a = 0, u32 b = 
   }
   st_u32(&c.ctl->stop, 2u);
 }
-__device__ __forceinline__ bool stopped(const Ctx &c) { return ld_u32(&c.ctl->stop) != 0u; }
 // warp-uniform variants: every lane gets lane 0's view, and the shuffle is a convergence point
 __device__ __forceinline__ bool warp_stopped(const Ctx &c) {
   return __shfl_sync(0xffffffffu, ld_u32(&c.ctl->stop), 0) != 0u;
@@ -1188,12 +1174,14 @@ __device__ void copy_page(const Ctx &c, u32 idx, u32 lane) {
   uint4 v[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) v[i] = __ldcs(src + i * 32 + lane);
-  // a value that depends on every loaded word: the acknowledgement cannot be issued early
-  u32 dep = 0;
+  // The acknowledgement carries a checksum of the page above the lap tag (the host looks at the
+  // tag only): a value that really depends on every loaded word, so the store cannot issue
+  // before the page's bytes have arrived.
+  u32 sum = 0;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) dep |= (v[i].x ^ v[i].x);
-  dep = __reduce_or_sync(0xffffffffu, dep);
-  if (lane == 0) st_sys_u32(c.fdone + (idx & c.ring_mask), ((u32)cmd & 0xFFu) | dep);
+  for (int i = 0; i < 8; ++i) sum ^= v[i].x ^ v[i].y ^ v[i].z ^ v[i].w;
+  sum = __reduce_xor_sync(0xffffffffu, sum);
+  if (lane == 0) st_sys_u32(c.fdone + (idx & c.ring_mask), ((u32)cmd & 0xFFu) | (sum << 8));
 #pragma unroll
   for (int i = 0; i < 8; ++i) __stcg(dst + i * 32 + lane, v[i]);
   __syncwarp();          // orders every lane's stores before lane 0's release below
