@@ -52,7 +52,7 @@ enum { GORIO_FLAG_PAGES_ALREADY_PINNED = 1u }; /* host_pages is already page-loc
  *   (cudaHostRegister) unless GORIO_FLAG_PAGES_ALREADY_PINNED is set.
  *   PQ navigation (optional): pq_m > 0 enables it; pq_centroids_dev is u8
  *   [pq_m][256][dim/pq_m] and pq_codes_dev is u8 [n_nodes][pq_m], both DEVICE memory
- *   borrowed until close.  Requires dtype u8, dim % pq_m == 0, (dim/pq_m) % 4 == 0.
+ *   borrowed until close.  Requires dtype u8, dim % pq_m == 0, dim/pq_m in {4, 8, 12, 16}.
  * Preconditions: page_bytes == 4096, dim % 4 == 0, nodes_per_page*node_bytes <= 4096,
  *   n_nodes < 2^31, entry_id < n_nodes, max_degree >= 1.
  */

@@ -371,7 +371,7 @@ int gorio_index_open(const gorio_index_desc *d, int cuda_device, gorio_index **o
     return GORIO_ERR_INVALID_ARG;
   if (d->pq_m) {
     if (d->dtype != GORIO_DTYPE_U8 || d->dim % d->pq_m != 0 || (d->dim / d->pq_m) % 4 != 0 ||
-        d->pq_m > 64 || !d->pq_centroids_dev || !d->pq_codes_dev)
+        d->pq_m > 64 || d->dim / d->pq_m > 16 || !d->pq_centroids_dev || !d->pq_codes_dev)
       return GORIO_ERR_INVALID_ARG;
   }
   gorio_index *ix = new (std::nothrow) gorio_index();
@@ -514,8 +514,8 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
     auto_warps = (nq + (u32)ix->n_sms - 1) / (u32)ix->n_sms;
     auto_warps = auto_warps < 8u ? 8u : (auto_warps > 24u ? 24u : auto_warps);
   }
-  u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 6u : auto_warps);
-  if (pq) { u32 lim = (200u * 1024u) / (d.pq_m * kPqKsub * 4u); if (warps > lim) warps = lim; }
+  u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 10u : auto_warps);
+  if (pq) { u32 lim = (220u * 1024u) / (d.pq_m * kPqLutWords * 4u); if (warps > lim) warps = lim; }
   if (warps < 2) return fail(ix, GORIO_ERR_INVALID_ARG, "search: need at least 2 warps per block (the poller and a worker)");
   int occ = 0;
   CK(search_occupancy(d.pq_m, warps, &occ));

@@ -17,6 +17,7 @@ constexpr u32 kClosed = 0xFFFFFFFEu;  // waiter list closed: the page has arrive
 constexpr u32 kInvalidId = 0xFFFFFFFFu;
 constexpr u64 kPadKey = ~0ull;        // sorts after every real key
 constexpr u32 kPqKsub = 256;
+constexpr u32 kPqLutWords = 160;       // u32 words of shared memory per subspace: 256 x u16 + 256 x 4 bits
 
 // Query phases: which batch of page items is outstanding for the query slot.
 enum Phase : u32 { PH_NEW = 0, PH_EVAL = 1, PH_EXPAND = 2 };

@@ -955,12 +955,23 @@ __device__ u32 collect_neighbors(const Ctx &c, u32 qs, u32 lane) {
 // ------------------------------------------------------------------------------------------
 // PQ asymmetric distance: per-query lookup table in shared memory
 // ------------------------------------------------------------------------------------------
-// LUT[m][c] = sum_j (q[m*dsub+j] - cent[m][c][j])^2 (u32, exact); adc(v) = sum_m LUT[m][code[v][m]]
+// LUT[m][c] = sum_j (q[m*dsub+j] - cent[m][c][j])^2 (exact, < 2^20 for dsub <= 16);
+// adc(v) = sum_m LUT[m][code[v][m]].
+// The table is stored losslessly in 20 bits per entry -- a u16 array of low halves followed by
+// the high nibbles packed eight to a word -- 640 bytes per subspace instead of 1024, so that
+// ten warps per SM can each keep a table instead of six.
+__device__ __forceinline__ const u32 *lut_hi(const Ctx &c, const u32 *lut) { return lut + c.pq_m * (kPqKsub / 2); }
+__device__ __forceinline__ u32 lut_get(const u16 *lo, const u32 *hi, u32 e) {
+  return (u32)lo[e] | (((hi[e >> 3] >> ((e & 7u) * 4u)) & 15u) << 16);
+}
+
 __device__ void build_lut(const Ctx &c, u32 qid, u32 *lut, u32 lane) {
   const u8 *q = (const u8 *)c.queries + (u64)qid * c.vec_bytes;
   const u32 wsub = c.pq_dsub >> 2;
   const u32 total = c.pq_m * kPqKsub;
-  for (u32 e = lane; e < total; e += 32) {
+  u16 *lo = (u16 *)lut;
+  u32 *hi = lut + c.pq_m * (kPqKsub / 2);
+  for (u32 e = lane; e < total; e += 32) {            // total is a multiple of 32: no lane idles
     const u32 m = e >> 8;
     const u32 *cw = (const u32 *)(c.pq_cent + (u64)e * c.pq_dsub);
     const u32 *qw = (const u32 *)(q + m * c.pq_dsub);
@@ -969,25 +980,27 @@ __device__ void build_lut(const Ctx &c, u32 qid, u32 *lut, u32 lane) {
       u32 d = __vabsdiffu4(__ldg(cw + w), __ldg(qw + w));
       s = __dp4a(d, d, s);
     }
-    lut[e] = s;
+    lo[e] = (u16)s;
+    // eight consecutive entries (lanes 8k..8k+7) share one word of high nibbles
+    u32 nib = ((s >> 16) & 15u) << ((lane & 7u) * 4u);
+    nib |= __shfl_xor_sync(0xffffffffu, nib, 1);
+    nib |= __shfl_xor_sync(0xffffffffu, nib, 2);
+    nib |= __shfl_xor_sync(0xffffffffu, nib, 4);
+    if ((lane & 7u) == 0) hi[e >> 3] = nib;
   }
   __syncwarp();
-}
-__device__ __forceinline__ u32 warp_adc(const Ctx &c, const u32 *lut, u32 v, u32 lane) {
-  u32 acc = 0;
-  const u8 *code = c.pq_codes + (u64)v * c.pq_m;
-  for (u32 m = lane; m < c.pq_m; m += 32) acc += lut[(m << 8) + __ldg(code + m)];
-  return __reduce_add_sync(0xffffffffu, acc);
 }
 // One node per lane: the lane reads the node's code (pq_m bytes, 4 at a time) and sums pq_m
 // independent table entries from shared memory -- no cross-lane reduction, 32 nodes per pass.
 __device__ __forceinline__ u32 lane_adc(const Ctx &c, const u32 *lut, u32 v) {
   const u32 *code = (const u32 *)(c.pq_codes + (u64)v * c.pq_m);
+  const u16 *lo = (const u16 *)lut;
+  const u32 *hi = lut_hi(c, lut);
   u32 acc = 0;
   for (u32 w = 0; w < (c.pq_m >> 2); ++w) {
     const u32 cw = __ldg(code + w);
-    acc += lut[((4u * w + 0u) << 8) + (cw & 255u)] + lut[((4u * w + 1u) << 8) + ((cw >> 8) & 255u)] +
-           lut[((4u * w + 2u) << 8) + ((cw >> 16) & 255u)] + lut[((4u * w + 3u) << 8) + (cw >> 24)];
+    acc += lut_get(lo, hi, ((4u * w + 0u) << 8) + (cw & 255u)) + lut_get(lo, hi, ((4u * w + 1u) << 8) + ((cw >> 8) & 255u)) +
+           lut_get(lo, hi, ((4u * w + 2u) << 8) + ((cw >> 16) & 255u)) + lut_get(lo, hi, ((4u * w + 3u) << 8) + (cw >> 24));
   }
   return acc;
 }
@@ -1109,8 +1122,7 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut, u32 &lut_qid
       __syncwarp();
       if (PQ) {
         if (lut_qid != qid) { build_lut(c, qid, lut, lane); lut_qid = qid; }
-        u32 d = warp_adc(c, lut, c.entry, lane);
-        if (lane == 0) st_u64(c.cand + (u64)qs * c.WR, mk_key(d, c.entry));
+        if (lane == 0) st_u64(c.cand + (u64)qs * c.WR, mk_key(lane_adc(c, lut, c.entry), c.entry));
         __syncwarp();
       } else {
         if (!issue_batch(c, qs, lane) && !(c.blocking && wait_in_place(c, qs, lane))) return;
@@ -1270,7 +1282,7 @@ __global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
   extern __shared__ u32 smem_lut[];
   const u32 lane = lane_id(), warp = threadIdx.x >> 5;
   if (blockIdx.x == 0 && warp == 0) { poller(c, lane); return; }
-  u32 *lut = PQ ? smem_lut + (u64)warp * c.pq_m * kPqKsub : nullptr;
+  u32 *lut = PQ ? smem_lut + (u64)warp * c.pq_m * kPqLutWords : nullptr;
   const u64 t0 = globaltimer();
   u32 idle = 0;
   // where the worker warps' time goes (ns, summed over warps): arrivals, query phases, idle
@@ -1385,11 +1397,11 @@ cudaError_t launch_cache_reset(const Ctx &c, u32 preloaded, cudaStream_t s) {
   return cudaGetLastError();
 }
 
-static size_t search_smem(const Ctx &c, u32 warps) { return c.pq_m ? (size_t)warps * c.pq_m * kPqKsub * 4 : 0; }
+static size_t search_smem(const Ctx &c, u32 warps) { return c.pq_m ? (size_t)warps * c.pq_m * kPqLutWords * 4 : 0; }
 
 cudaError_t search_occupancy(u32 pq_m, u32 warps_per_block, int *blocks_per_sm) {
   if (pq_m) {
-    const size_t smem = (size_t)warps_per_block * pq_m * kPqKsub * 4;
+    const size_t smem = (size_t)warps_per_block * pq_m * kPqLutWords * 4;
     cudaError_t e = cudaFuncSetAttribute(search_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<true>, warps_per_block * 32, smem);
