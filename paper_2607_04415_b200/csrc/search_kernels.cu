@@ -753,33 +753,41 @@ __device__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
 // Bitonic sort of 32*NPL u64 keys held NPL per lane, element e at lane e%32, register e/32.
 template <int NPL>
 __device__ __forceinline__ void bitonic_sort(u64 (&x)[NPL], u32 lane) {
+  // Stages whose stride is below 32 exchange between lanes and do the same thing to every
+  // register, so they run as a runtime loop over one stage body; stages with a stride of 32 or
+  // more pair registers and need static indices.  (Fully unrolled, the 512-key network is
+  // several thousand instructions, and warps in different phases evict each other's code.)
+#pragma unroll 1
+  for (u32 k = 2; k <= 32u * NPL; k <<= 1) {
 #pragma unroll
-  for (int k = 2; k <= 32 * NPL; k <<= 1) {
+    for (int kk = 64; kk <= 32 * NPL; kk <<= 1) {
+      if (k == (u32)kk) {
 #pragma unroll
-    for (int j = k >> 1; j > 0; j >>= 1) {
-      if (j >= 32) {
-        const int jr = j >> 5;
+        for (int jr = kk >> 6; jr > 0; jr >>= 1) {
 #pragma unroll
-        for (int r = 0; r < NPL; ++r) {
-          const int pr = r ^ jr;
-          if (pr > r) {
-            const bool asc = ((r << 5) & k) == 0;
-            const u64 a = x[r], b = x[pr];
-            const bool sw = asc ? (a > b) : (a < b);
-            x[r] = sw ? b : a;
-            x[pr] = sw ? a : b;
+          for (int r = 0; r < NPL; ++r) {
+            const int pr = r ^ jr;
+            if (pr > r) {
+              const bool asc = ((r << 5) & kk) == 0;
+              const u64 a = x[r], b = x[pr];
+              const bool sw = asc ? (a > b) : (a < b);
+              x[r] = sw ? b : a;
+              x[pr] = sw ? a : b;
+            }
           }
         }
-      } else {
+      }
+    }
+#pragma unroll 1
+    for (u32 j = (k >> 1) < 16u ? (k >> 1) : 16u; j > 0; j >>= 1) {
+      const bool lower = (lane & j) == 0;
 #pragma unroll
-        for (int r = 0; r < NPL; ++r) {
-          const u64 a = x[r];
-          const u64 b = __shfl_xor_sync(0xffffffffu, a, j);
-          const bool asc = ((((u32)r << 5) | lane) & (u32)k) == 0;
-          const bool lower = (lane & (u32)j) == 0;
-          const u64 mn = a < b ? a : b, mx = a < b ? b : a;
-          x[r] = (asc == lower) ? mn : mx;
-        }
+      for (int r = 0; r < NPL; ++r) {
+        const u64 a = x[r];
+        const u64 b = __shfl_xor_sync(0xffffffffu, a, j);
+        const bool asc = ((((u32)r << 5) | lane) & k) == 0;
+        const u64 mn = a < b ? a : b, mx = a < b ? b : a;
+        x[r] = (asc == lower) ? mn : mx;
       }
     }
   }
