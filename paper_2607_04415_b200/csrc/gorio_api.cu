@@ -151,10 +151,22 @@ void proxy_service(gorio_index *ix) {
   std::deque<InService> inflight;
   u64 fetched = 0, max_seen = 0, batches = 0;
   u64 service_ns = 0, ack_wait_iters = 0, window_full_iters = 0, ring_empty_iters = 0, iters = 0, out_sum = 0;
+  // debug aid (with GORIO_CENSUS_MS): fetches published and mean outstanding per 10 ms interval
+  const bool trace = std::getenv("GORIO_CENSUS_MS") != nullptr;
+  std::vector<u64> tr_fetched, tr_out;
+  Clock::time_point tr_next = Clock::now() + std::chrono::milliseconds(10);
+  u64 tr_out_sum = 0, tr_iters = 0;
 
   while (!ix->px_stop.load(std::memory_order_acquire)) {
     ++iters;
     out_sum += outstanding;
+    if (trace) {
+      tr_out_sum += outstanding; ++tr_iters;
+      if ((iters & 63) == 0 && Clock::now() >= tr_next) {
+        tr_fetched.push_back(fetched); tr_out.push_back(tr_out_sum / (tr_iters ? tr_iters : 1));
+        tr_out_sum = tr_iters = 0; tr_next += std::chrono::milliseconds(10);
+      }
+    }
     // 1. admit descriptors while the in-service window has room; each becomes a copy command
     u32 admitted = 0;
     const Clock::time_point now0 = Clock::now();
@@ -198,6 +210,12 @@ void proxy_service(gorio_index *ix) {
         fetched += published;
       }
     }
+  }
+  if (trace) {
+    std::fprintf(stderr, "[gorio proxy] per 10 ms: fetched(k)/mean outstanding:");
+    u64 prev = 0;
+    for (size_t i = 0; i < tr_fetched.size(); ++i) { std::fprintf(stderr, " %llu/%llu", (unsigned long long)((tr_fetched[i] - prev) / 1000), (unsigned long long)tr_out[i]); prev = tr_fetched[i]; }
+    std::fprintf(stderr, "\n");
   }
   ix->px_dbg[0] = tail; ix->px_dbg[1] = ct; ix->px_dbg[2] = outstanding; ix->px_dbg[3] = (u32)inflight.size();
   if (!inflight.empty()) {
