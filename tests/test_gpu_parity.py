@@ -1,6 +1,8 @@
 """GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, element by
 element on the same seeded inputs.  uint8 data must match bit-exactly (ids, integer
 distances, per-query counters); fp32 within the tolerance procedure below."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -412,3 +414,34 @@ def test_second_search_reuses_the_warm_cache(gorio, cfg1):
         assert f1 == int(ref["page_union"].sum()) and f2 == 0
     finally:
         ix.close()
+
+
+# ------------------------------------------------------------------ randomized configurations
+@pytest.mark.parametrize("seed", list(range(int(os.environ.get("GORIO_FUZZ_SEEDS", "24")))))
+def test_randomized_configurations_match_oracle(gorio, seed):
+    """Small random indexes under random search, cache, proxy and scheduler settings: whatever
+    the interleaving of misses, arrivals, evictions and resumes, uint8 results are bit-exact."""
+    from workloads import node_bytes as nbytes
+    rng = np.random.default_rng(1000 + seed)
+    d = int(rng.choice([16, 32, 48, 64, 128]))
+    R = int(rng.integers(4, 33))
+    nb = nbytes(d, np.uint8, R)
+    npp = int(rng.integers(1, 4096 // nb + 1))
+    N = int(rng.integers(400, 5000))
+    C = int(rng.integers(1, 6))
+    nq = int(rng.integers(1, 500))
+    k = int(rng.integers(2, R))
+    L = int(rng.integers(4, 129))
+    W = int(rng.integers(1, min(9, 1024 // R)))
+    K = int(rng.integers(1, min(L, 20) + 1))
+    w = make_workload(f"rnd{seed}", "u8", N, C, nq, d, k, R - k, npp, clustered_knn=bool(rng.integers(0, 2)),
+                      cross_only=False, with_gt=False, K=K, L=L, W=W)
+    ref = OracleIndex.from_workload(w).search(w.queries, K, L, W, threads=4)
+    cap = int(rng.integers(16, max(17, w.n_pages + 1)))
+    tuning = dict(warps_per_block=int(rng.integers(2, 17)), max_inflight=int(rng.choice([0, 8, 64])),
+                  stash_entries=int(rng.choice([0, 1, 64, 256])), blocking=int(rng.integers(0, 2)),
+                  request_backlog=int(rng.choice([0, 1, 16, 4096])))
+    got = _gpu_search(gorio, w, cap, K=K, L=L, W=W, tuning=tuning, preload=bool(rng.integers(0, 4) == 0),
+                      remote_latency_ns=int(rng.choice([0, 2000, 20000])), max_outstanding=int(rng.choice([1, 8, 256])))
+    _assert_exact(got, ref)
+    assert got["stats"]["queries_done"] == nq
