@@ -445,3 +445,31 @@ def test_randomized_configurations_match_oracle(gorio, seed):
                       remote_latency_ns=int(rng.choice([0, 2000, 20000])), max_outstanding=int(rng.choice([1, 8, 256])))
     _assert_exact(got, ref)
     assert got["stats"]["queries_done"] == nq
+
+
+@pytest.mark.parametrize("seed", list(range(8)))
+def test_randomized_fp32_and_pq_configurations(gorio, seed):
+    from workloads import node_bytes as nbytes
+    rng = np.random.default_rng(5000 + seed)
+    pq = seed % 2 == 1
+    R = int(rng.integers(6, 25))
+    if pq:
+        kind, d = "u8", int(rng.choice([32, 64, 128]))          # 8 / 16 / 32 ... subspaces of 4 bytes
+    else:
+        kind, d = "f32", int(rng.choice([8, 24, 40, 96]))
+    nb = nbytes(d, np.uint8 if kind == "u8" else np.float32, R)
+    npp = int(rng.integers(1, 4096 // nb + 1))
+    N, nq = int(rng.integers(1500, 6000)), int(rng.integers(20, 300))
+    L, W = int(rng.integers(16, 100)), int(rng.integers(1, 6))
+    w = make_workload(f"rnd{seed}", kind, N, 4, nq, d, R - 3, 3, npp, clustered_knn=True, cross_only=False,
+                      with_gt=not pq, K=8, L=L, W=W)
+    if pq:
+        w.pq_centroids, w.pq_codes = train_pq(w.data, m=d // 4, sample=2048, iters=3)
+    ref = OracleIndex.from_workload(w, use_pq=pq).search(w.queries, 8, L, W, threads=4)
+    cap = int(rng.integers(16, max(17, w.n_pages // 2)))
+    got = _gpu_search(gorio, w, cap, K=8, L=L, W=W, use_pq=pq, remote_latency_ns=int(rng.choice([0, 5000])),
+                      max_outstanding=int(rng.choice([4, 256])), tuning=dict(max_inflight=int(rng.choice([0, 32]))))
+    if pq:
+        _assert_exact(got, ref)
+    else:
+        _fp32_parity(w, got, ref)
