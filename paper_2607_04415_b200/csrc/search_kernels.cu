@@ -751,14 +751,16 @@ __device__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
 // warp-sorted candidate list
 // ------------------------------------------------------------------------------------------
 // Bitonic sort of 32*NPL u64 keys held NPL per lane, element e at lane e%32, register e/32.
+// k_first = 2 sorts; k_first = 32*NPL runs only the last pass, which merges an array whose
+// lower half ascends and whose upper half descends.  desc sorts into descending order.
 template <int NPL>
-__device__ __forceinline__ void bitonic_sort(u64 (&x)[NPL], u32 lane) {
+__device__ __forceinline__ void bitonic_sort(u64 (&x)[NPL], u32 lane, u32 k_first = 2, bool desc = false) {
   // Stages whose stride is below 32 exchange between lanes and do the same thing to every
   // register, so they run as a runtime loop over one stage body; stages with a stride of 32 or
   // more pair registers and need static indices.  (Fully unrolled, the 512-key network is
   // several thousand instructions, and warps in different phases evict each other's code.)
 #pragma unroll 1
-  for (u32 k = 2; k <= 32u * NPL; k <<= 1) {
+  for (u32 k = k_first; k <= 32u * NPL; k <<= 1) {
 #pragma unroll
     for (int kk = 64; kk <= 32 * NPL; kk <<= 1) {
       if (k == (u32)kk) {
@@ -768,7 +770,7 @@ __device__ __forceinline__ void bitonic_sort(u64 (&x)[NPL], u32 lane) {
           for (int r = 0; r < NPL; ++r) {
             const int pr = r ^ jr;
             if (pr > r) {
-              const bool asc = ((r << 5) & kk) == 0;
+              const bool asc = (((r << 5) & kk) == 0) != desc;
               const u64 a = x[r], b = x[pr];
               const bool sw = asc ? (a > b) : (a < b);
               x[r] = sw ? b : a;
@@ -785,7 +787,7 @@ __device__ __forceinline__ void bitonic_sort(u64 (&x)[NPL], u32 lane) {
       for (int r = 0; r < NPL; ++r) {
         const u64 a = x[r];
         const u64 b = __shfl_xor_sync(0xffffffffu, a, j);
-        const bool asc = ((((u32)r << 5) | lane) & k) == 0;
+        const bool asc = (((((u32)r << 5) | lane) & k) == 0) != desc;
         const u64 mn = a < b ? a : b, mx = a < b ? b : a;
         x[r] = (asc == lower) ? mn : mx;
       }
@@ -811,7 +813,12 @@ __device__ __noinline__ u32 merge_select(const Ctx &c, u32 qs, u32 lane) {
   const u32 nc = uld(&h->n_items);
   u64 *list = c.list + (u64)qs * c.L;
   const u64 *cand = c.cand + (u64)qs * c.WR;
-  constexpr u32 CAP = 32u * NPL;
+  // The list (sorted, at most L <= 16*NPL keys) lives in the lower half of the registers.  A
+  // chunk of up to 16*NPL new candidates is sorted on its own, descending, in the upper half,
+  // which makes the whole array bitonic; one merge pass then orders it, and everything beyond
+  // L is dropped.  (Sorting list and candidates together cost 2-4x the compare-exchanges.)
+  constexpr int H = NPL / 2;
+  constexpr u32 HALF = 16u * NPL;
   u64 x[NPL];
 #pragma unroll
   for (int r = 0; r < NPL; ++r) {
@@ -820,15 +827,24 @@ __device__ __noinline__ u32 merge_select(const Ctx &c, u32 qs, u32 lane) {
   }
   u32 done = 0;
   while (done < nc) {
-    const u32 take = min(CAP - len, nc - done);
+    const u32 take = min(HALF, nc - done);
+    u64 y[H];
+#pragma unroll
+    for (int r = 0; r < H; ++r) {
+      const u32 e = (u32)r * 32u + lane;
+      y[r] = e < take ? ld_u64(cand + done + e) : kPadKey;
+    }
+    bitonic_sort<H>(y, lane, 2, true);
+#pragma unroll
+    for (int r = 0; r < H; ++r) x[H + r] = y[r];
+    bitonic_sort<NPL>(x, lane, 32u * NPL);
+    len = min(c.L, len + take);
+    done += take;
 #pragma unroll
     for (int r = 0; r < NPL; ++r) {
       const u32 e = (u32)r * 32u + lane;
-      if (e >= len) x[r] = (e - len < take) ? ld_u64(cand + done + (e - len)) : kPadKey;
+      if (e >= len) x[r] = kPadKey;
     }
-    bitonic_sort<NPL>(x, lane);
-    len = min(c.L, len + take);
-    done += take;
   }
   // frontier
   u32 taken = 0;
@@ -870,9 +886,9 @@ __device__ __noinline__ u32 merge_select(const Ctx &c, u32 qs, u32 lane) {
 }
 
 __device__ u32 merge_select_dispatch(const Ctx &c, u32 qs, u32 lane) {
-  const u32 need = c.L + c.WR;
-  if (need <= 128) return merge_select<4>(c, qs, lane);
-  if (need <= 256) return merge_select<8>(c, qs, lane);
+  if (c.L <= 32) return merge_select<2>(c, qs, lane);        // the list fits half of 32*NPL keys
+  if (c.L <= 64) return merge_select<4>(c, qs, lane);
+  if (c.L <= 128) return merge_select<8>(c, qs, lane);
   return merge_select<16>(c, qs, lane);
 }
 
