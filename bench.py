@@ -123,6 +123,8 @@ def main():
     ap.add_argument("--sweep", default=None,
                     help="comma list of latency_us:max_outstanding points; prints one short JSON line per point "
                          "(characterisation runs, not the benchmark line)")
+    ap.add_argument("--granularity", default="page", choices=["page", "record"],
+                    help="record: selective materialisation, a miss fetches only the wanted node's record")
     ap.add_argument("--L", type=int, default=None)
     ap.add_argument("--W", type=int, default=None)
     args = ap.parse_args()
@@ -203,7 +205,7 @@ def main():
 
     def reset_cache():
         ix.cache_config(cap, remote_latency_ns=lat_ns, max_outstanding=max_out, preload=preload,
-                        timeout_ms=120_000)
+                        timeout_ms=120_000, granularity=args.granularity)
         ix.stats_reset()
         l2_flush(flush)
 
@@ -231,14 +233,14 @@ def main():
                     ts.append(t); sts.append(st_i)
             ms_p = statistics.mean(ts)
             f_p = statistics.mean(x["pages_fetched"] for x in sts)
-            terms_p = {"host_link": 4096 * f_p / (h2d * 1e9), "outstanding_window": f_p * lat_ns * 1e-9 / max_out}
+            terms_p = {"host_link": statistics.mean(x["fetched_bytes"] for x in sts) / (h2d * 1e9), "outstanding_window": f_p * lat_ns * 1e-9 / max_out}
             bound_p = max(terms_p, key=terms_p.get)
             if rank == 0:
                 print(json.dumps({"latency_us": float(lat_us), "max_outstanding": max_out, "qps": world * w.nq / (ms_p * 1e-3),
                                   "ms_per_step": ms_p, "pages_fetched": f_p, "fetch_rate_M_per_s": f_p / ms_p / 1e3,
                                   "bound": bound_p, "frac": terms_p[bound_p] / (ms_p * 1e-3),
                                   "service_us": statistics.mean(x["proxy_service_ns"] / max(1, x["pages_fetched"]) for x in sts) / 1e3,
-                                  "blocking": bool(args.blocking)}))
+                                  "blocking": bool(args.blocking), "granularity": args.granularity}))
         ix.close()
         return
     for _ in range(max(3, args.warmup)):
@@ -266,6 +268,7 @@ def main():
     ms = statistics.mean(times)
     st = stats_list[len(stats_list) // 2]
     fetched = statistics.mean(s["pages_fetched"] for s in stats_list)
+    fetched_bytes = statistics.mean(s["fetched_bytes"] for s in stats_list)   # 4096 per page, or the record span
     launches = 2 * len(stats_list)          # init + persistent search kernel per step
 
     # roofline: the slowest of (a) algorithmic HBM bytes at the measured copy peak, (b) fetched
@@ -275,9 +278,9 @@ def main():
         b_alg = st["n_eval"] * 32 + st["n_expand"] * w.node_bytes
     else:
         b_alg = st["n_eval"] * w.d * esz + 4 * st["n_expand"] + 4 * st["sum_degree"]
-    b_hbm = b_alg + 4096 * fetched
+    b_hbm = b_alg + fetched_bytes
     t_a = b_hbm / (pk["hbm_gbs"] * 1e9)
-    t_b = 4096 * fetched / (h2d * 1e9)
+    t_b = fetched_bytes / (h2d * 1e9)
     t_c = fetched * lat_ns * 1e-9 / max_out
     terms = {"hbm": t_a, "host_link": t_b, "outstanding_window": t_c}
     bound = max(terms, key=terms.get)
@@ -285,13 +288,13 @@ def main():
     if bound == "hbm":
         ach, peak, unit = b_hbm / (ms * 1e-3) / 1e9, pk["hbm_gbs"], "GB/s"
     elif bound == "host_link":
-        ach, peak, unit = 4096 * fetched / (ms * 1e-3) / 1e9, h2d, "GB/s"
+        ach, peak, unit = fetched_bytes / (ms * 1e-3) / 1e9, h2d, "GB/s"
     else:
         ach, peak, unit = fetched / (ms * 1e-3) / 1e6, max_out / max(lat_ns * 1e-9, 1e-12) / 1e6, "Mfetch/s"
 
     default_workload = (args.config == 3 and args.scale == 1.0 and args.nq is None and not args.preload and
                         not args.blocking and args.cache_frac == 0.20 and args.latency_us is None and
-                        not args.max_outstanding and not args.L and not args.W)
+                        not args.max_outstanding and not args.L and not args.W and args.granularity == "page")
     ids = out["ids"].cpu().numpy().view(np.uint32)
     recall = recall_at_k(ids, w.gt)
     line = {
@@ -301,7 +304,8 @@ def main():
         "config": {"workload": f"cfg{args.config}{' SIFT1M-shaped' if args.config == 3 else ''}: N={w.N} d={w.d} {w.dtype} "
                                f"R={w.R} npp={w.npp} pages={w.n_pages} nq={w.nq}/gpu K={w.K} L={w.L} W={w.W} "
                                f"cache={cap} slots {'preloaded' if preload else 'cold'} latency={w.latency_us:g}us "
-                               f"max_outstanding={max_out}{' PQ 32x256' if args.config == 4 else ''}{' BLOCKING ablation' if args.blocking else ''}",
+                               f"max_outstanding={max_out}{' PQ 32x256' if args.config == 4 else ''}{' BLOCKING ablation' if args.blocking else ''}"
+                               f"{' RECORD granularity (selective materialisation)' if args.granularity == 'record' else ''}",
                    "recall_at_10": recall, "l2": "flushed before every step (512 MB read+write)",
                    "cache": "re-created cold before every step, untimed", "parallelism": f"query-sharded x{world}",
                    "context": PAPER_CONTEXT},
@@ -313,7 +317,7 @@ def main():
         "roofline": {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": t_roof / (ms * 1e-3),
                      "traffic": (NCU_DRAM_BYTES_PER_LAUNCH_CFG3 if default_workload else None), "peak_kind": f"hbm {pk_kind}; host link measured in this run ({h2d:.1f} GB/s)",
                      "terms_ms": {k: 1e3 * v for k, v in terms.items()},
-                     "pages_fetched": fetched, "algorithmic_hbm_bytes": b_hbm,
+                     "pages_fetched": fetched, "fetched_bytes": fetched_bytes, "algorithmic_hbm_bytes": b_hbm,
                      "hbm_achieved_gbs": b_hbm / (ms * 1e-3) / 1e9, "hbm_peak_gbs": pk["hbm_gbs"]},
         "stats": {k: st[k] for k in ("pages_hit", "pages_missed", "pages_fetched", "dedupe_joins", "evictions",
                                      "retries", "max_outstanding_seen", "resumes", "proxy_batches", "proxy_service_ns",

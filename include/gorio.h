@@ -84,6 +84,17 @@ typedef struct {
  *   preload          1: fill the cache with pages 0..capacity-1 now (whole index when
  *                    capacity >= n_pages); 0: start cold.
  *   timeout_ms       bound on one gorio_search call (device and host waits); 0 = 60000.
+ *   granularity      GORIO_GRAN_PAGE (0): a miss fetches the whole 4 KB page and a slot holds a
+ *                    page.  GORIO_GRAN_RECORD (1): selective materialisation (Section 7.2,
+ *                    third direction: return only the graph records that are needed instead of
+ *                    whole pages): a miss fetches just the wanted node's record -- the
+ *                    16-byte-aligned span of the page that covers it, node_bytes + 12 rounded
+ *                    up to 16 (400 bytes for a 388-byte record) -- and the cache holds records:
+ *                    capacity_pages * 4096 bytes of HBM are divided into record slots (capped
+ *                    at one slot per node), the lookup table has one word per node.  Search
+ *                    results and per-query counters are identical in both modes (pages_distinct
+ *                    still counts index pages); only the number and size of remote reads
+ *                    change.  preload must be 0 in this mode.
  * The proxy moves a page by writing a copy command into host-mapped memory; warps of the
  * search kernel pull the page from the pinned store into its slot and acknowledge, and the
  * proxy publishes the completion after the latency.  No CUDA call is made while a search runs.
@@ -95,9 +106,11 @@ typedef struct {
   uint32_t max_outstanding;
   uint32_t preload;
   uint32_t timeout_ms;
-  uint32_t reserved0;
+  uint32_t granularity;
   uint32_t reserved1;
 } gorio_cache_cfg;
+
+enum { GORIO_GRAN_PAGE = 0, GORIO_GRAN_RECORD = 1 };
 
 /*
  * Scheduler tuning; all zero = defaults.
@@ -131,7 +144,8 @@ typedef struct {
  * Counters since the last gorio_stats_reset.
  *   pages_hit      page lookups satisfied from a resident slot
  *   pages_missed   (query, node) waits registered on a page in flight (owner or joiner)
- *   pages_fetched  request descriptors the proxy serviced (4 KB each)
+ *   pages_fetched  request descriptors the proxy serviced (4 KB each; one record each at
+ *                  record granularity); fetched_bytes: the bytes they moved over the host link
  *   dedupe_joins   waits that joined another query's or lane's outstanding request
  *   evictions, retries (hits that were evicted under the read and looked up again),
  *   max_outstanding_seen (proxy), queries_done,
@@ -154,6 +168,7 @@ typedef struct {
      running query phases, idle; the number of arrival-queue items consumed; ns executing copy commands */
   uint64_t warp_ns_arrivals, warp_ns_queries, warp_ns_idle, arrivals_consumed;
   uint64_t warp_ns_copies, stash_hits;   /* expansions served from the adjacency stash */
+  uint64_t fetched_bytes;
 } gorio_stats_t;
 
 /* Open an index on CUDA device `cuda_device`.  *out is set only on GORIO_OK. */

@@ -38,7 +38,7 @@ class _IndexDesc(ctypes.Structure):
 class _CacheCfg(ctypes.Structure):
     _fields_ = [("capacity_pages", ctypes.c_uint64), ("remote_latency_ns", ctypes.c_uint32),
                 ("max_outstanding", ctypes.c_uint32), ("preload", ctypes.c_uint32),
-                ("timeout_ms", ctypes.c_uint32), ("reserved0", ctypes.c_uint32),
+                ("timeout_ms", ctypes.c_uint32), ("granularity", ctypes.c_uint32),
                 ("reserved1", ctypes.c_uint32)]
 
 
@@ -54,7 +54,7 @@ _STAT_FIELDS = ["pages_hit", "pages_missed", "pages_fetched", "dedupe_joins", "e
                 "resumes", "search_ns", "proxy_batches", "posted", "proxy_service_ns", "proxy_iters",
                 "proxy_ack_wait_iters", "proxy_window_full_iters", "proxy_ring_empty_iters",
                 "proxy_outstanding_sum", "warp_ns_arrivals", "warp_ns_queries", "warp_ns_idle",
-                "arrivals_consumed", "warp_ns_copies", "stash_hits"]
+                "arrivals_consumed", "warp_ns_copies", "stash_hits", "fetched_bytes"]
 
 
 class Stats(ctypes.Structure):
@@ -146,9 +146,11 @@ class Index:
             raise GorioError(status, detail or self._lib.gorio_status_str(status).decode())
 
     def cache_config(self, capacity_pages, remote_latency_ns=0, max_outstanding=256, preload=False,
-                     timeout_ms=0):
+                     timeout_ms=0, granularity="page"):
+        """granularity: "page" (a miss fetches the 4 KB page) or "record" (only the wanted node's record)."""
+        gran = {"page": 0, "record": 1}[granularity]
         cfg = _CacheCfg(int(capacity_pages), int(remote_latency_ns), int(max_outstanding), int(bool(preload)),
-                        int(timeout_ms), 0, 0)
+                        int(timeout_ms), gran, 0)
         self._check(self._lib.gorio_cache_config(self._h, ctypes.byref(cfg)))
 
     def set_tuning(self, max_inflight=0, visited_capacity=0, warps_per_block=0, blocks_per_sm=0, stash_entries=0,

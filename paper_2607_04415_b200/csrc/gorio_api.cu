@@ -43,6 +43,7 @@ struct gorio_index {
   gorio_cache_cfg cfg{};
   bool cache_ready = false, cache_dirty = false;
   u32 n_slots = 0, preloaded = 0;
+  u32 n_units = 0, slot_bytes = kPageBytes, record_mode = 0;   // cache unit: page, or node record
   u8 *slot_data = nullptr;
   u64 *ptab = nullptr, *smeta = nullptr;
   u32 *parts = nullptr, *filled = nullptr;
@@ -57,7 +58,7 @@ struct gorio_index {
 
   // query state
   gorio_tuning tune{};
-  u32 qs_slots = 0, qs_L = 0, qs_W = 0, qs_WR = 0, qs_K = 0, qs_seen = 0, qs_pset = 0, qs_stash = 0, qs_nslots = 0;
+  u32 qs_slots = 0, qs_L = 0, qs_W = 0, qs_WR = 0, qs_K = 0, qs_seen = 0, qs_pset = 0, qs_stash = 0, qs_nslots = 0, qs_units = 0;
   void *qs_block = nullptr;
   Ctx ctx{};
   Ctl *ctl = nullptr;
@@ -78,6 +79,7 @@ struct gorio_index {
   cudaEvent_t done_ev = nullptr;
 
   // statistics
+  u64 host_fetched_bytes = 0;
   u64 host_fetched = 0, host_max_out = 0, host_batches = 0, host_search_ns = 0;
   u64 host_service_ns = 0, host_ack_wait = 0, host_window_full = 0, host_ring_empty = 0, host_iters = 0, host_out_sum = 0;
   u32 px_dbg[8] = {};   // proxy progress at the end of its last service loop
@@ -175,7 +177,7 @@ void proxy_service(gorio_index *ix) {
       const u32 lap = ((tail >> ring_shift) % 255u) + 1u;
       if ((u32)(e & 0xFFu) != lap) break;
       const u32 page = (u32)(e >> 32), slot = (u32)(e >> 8) & 0xFFFFFFu;
-      if (page >= ix->n_pages || slot >= ix->n_slots) {
+      if (page >= ix->n_units || slot >= ix->n_slots) {
         ix->px_error.store(1);   // a descriptor the GPU could not have produced
         return;
       }
@@ -225,6 +227,7 @@ void proxy_service(gorio_index *ix) {
   ix->host_service_ns += service_ns; ix->host_ack_wait += ack_wait_iters; ix->host_window_full += window_full_iters;
   ix->host_ring_empty += ring_empty_iters; ix->host_iters += iters; ix->host_out_sum += out_sum;
   ix->host_fetched += fetched;
+  ix->host_fetched_bytes += fetched * ix->slot_bytes;
   ix->host_batches += batches;
   if (max_seen > ix->host_max_out) ix->host_max_out = max_seen;
 }
@@ -266,12 +269,22 @@ void proxy_stop(gorio_index *ix) {
 int setup_cache(gorio_index *ix) {
   const gorio_cache_cfg &cfg = ix->cfg;
   free_cache(ix);
-  const u64 cap = cfg.capacity_pages;
-  ix->n_slots = cap >= ix->n_pages ? ix->n_pages : (u32)cap;
+  u64 cap = cfg.capacity_pages;
+  ix->record_mode = cfg.granularity == GORIO_GRAN_RECORD ? 1u : 0u;
+  if (ix->record_mode) {
+    // selective materialisation: the same bytes of HBM, divided into record-sized slots
+    ix->n_units = (u32)ix->desc.n_nodes;
+    ix->slot_bytes = (ix->node_bytes + 12u + 15u) & ~15u;
+    cap = cap * kPageBytes / ix->slot_bytes;
+  } else {
+    ix->n_units = ix->n_pages;
+    ix->slot_bytes = kPageBytes;
+  }
+  ix->n_slots = cap >= ix->n_units ? ix->n_units : (u32)cap;
   ix->ring_cap = next_pow2(2ull * ix->n_slots < 1024 ? 1024 : 2ull * ix->n_slots);
-  ix->want_cap = next_pow2(ix->n_pages < 64 ? 64 : ix->n_pages);
-  CK(cudaMalloc(&ix->slot_data, (size_t)ix->n_slots * kPageBytes));
-  CK(cudaMalloc(&ix->ptab, (size_t)ix->n_pages * 8));
+  ix->want_cap = next_pow2(ix->n_units < 64 ? 64 : ix->n_units);
+  CK(cudaMalloc(&ix->slot_data, (size_t)ix->n_slots * ix->slot_bytes));
+  CK(cudaMalloc(&ix->ptab, (size_t)ix->n_units * 8));
   CK(cudaMalloc(&ix->smeta, (size_t)ix->n_slots * 8));
   CK(cudaMalloc(&ix->parts, (size_t)ix->n_slots * 4));
   CK(cudaMalloc(&ix->filled, (size_t)ix->n_slots * 4));
@@ -287,7 +300,7 @@ int setup_cache(gorio_index *ix) {
   }
   Ctx c{};
   c.ptab = ix->ptab; c.smeta = ix->smeta; c.parts = ix->parts; c.filled = ix->filled; c.cs = ix->cs;
-  c.n_slots = ix->n_slots; c.n_pages = ix->n_pages;
+  c.n_slots = ix->n_slots; c.n_pages = ix->n_pages; c.n_units = ix->n_units;
   CK(launch_cache_reset(c, ix->preloaded, ix->own_stream));
   CK(cudaStreamSynchronize(ix->own_stream));
   ix->cache_ready = true;
@@ -303,7 +316,7 @@ int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W) {
   const u32 pset_cap = ix->desc.pq_m ? 4096u : seen_cap;
   if (ix->qs_block && ix->qs_slots >= slots && ix->qs_L == L && ix->qs_W == W && ix->qs_K == K &&
       ix->qs_seen == seen_cap && ix->qs_pset == pset_cap && ix->qs_stash == (ix->tune.stash_entries + 1u) &&
-      ix->qs_nslots == ix->n_slots) {      // (the arrival queue and the stash default depend on the slot count)
+      ix->qs_nslots == ix->n_slots && ix->qs_units == ix->n_units) {      // (the arrival queue and the stash default depend on the slot count)
     ix->ctx.n_qslots = slots;
     return GORIO_OK;
   }
@@ -323,7 +336,7 @@ int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W) {
   // adjacency stash: exact navigation only; by default on (1024 entries) unless every page has
   // a slot of its own, in which case expansions seldom wait for a page and the copies are waste
   u32 stash_cap = ix->tune.stash_entries > 1 ? ix->tune.stash_entries
-                  : (ix->tune.stash_entries == 1 || ix->n_slots >= ix->n_pages ? 0u : 1024u);
+                  : (ix->tune.stash_entries == 1 || ix->n_slots >= ix->n_units ? 0u : 1024u);
   if (ix->desc.pq_m) stash_cap = 0;
   const size_t o_stag = off; off += al((size_t)slots * stash_cap * 4);
   const size_t o_stash = off; off += al((size_t)slots * stash_cap * (R + 1) * 4);
@@ -342,6 +355,7 @@ int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W) {
   c.seen_cap = seen_cap; c.pset_cap = pset_cap; c.n_qslots = slots;
   ix->qs_slots = slots; ix->qs_L = L; ix->qs_W = W; ix->qs_WR = WR; ix->qs_K = K;
   ix->qs_seen = seen_cap; ix->qs_pset = pset_cap; ix->qs_stash = ix->tune.stash_entries + 1u; ix->qs_nslots = ix->n_slots;
+  ix->qs_units = ix->n_units;
   return GORIO_OK;
 }
 
@@ -454,7 +468,14 @@ int gorio_cache_config(gorio_index *ix, const gorio_cache_cfg *cfg) {
   if (!ix || !cfg) return GORIO_ERR_INVALID_ARG;
   if (cfg->capacity_pages < 16 || cfg->max_outstanding < 1)
     return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: capacity >= 16, max_outstanding >= 1");
+  if (cfg->granularity > GORIO_GRAN_RECORD) return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: unknown granularity");
+  if (cfg->granularity == GORIO_GRAN_RECORD && cfg->preload)
+    return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: preload needs page granularity");
   u64 cap = cfg->capacity_pages < ix->n_pages ? cfg->capacity_pages : ix->n_pages;
+  if (cfg->granularity == GORIO_GRAN_RECORD) {
+    cap = cap * kPageBytes / ((ix->node_bytes + 12u + 15u) & ~15u);
+    if (cap > ix->desc.n_nodes) cap = ix->desc.n_nodes;
+  }
   if (cap >= (1ull << 24)) return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: at most 2^24 slots");
   CK(cudaSetDevice(ix->dev));
   ix->cfg = *cfg;
@@ -497,7 +518,7 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   c.node_bytes = ix->node_bytes; c.vec_bytes = ix->vec_bytes; c.entry = d.entry_id; c.n_pages = ix->n_pages;
   c.pq_m = d.pq_m; c.pq_dsub = d.pq_m ? d.dim / d.pq_m : 0; c.pq_cent = d.pq_centroids_dev; c.pq_codes = d.pq_codes_dev;
   c.slot_data = ix->slot_data; c.ptab = ix->ptab; c.smeta = ix->smeta; c.parts = ix->parts; c.filled = ix->filled; c.cs = ix->cs;
-  c.n_slots = ix->n_slots;
+  c.n_slots = ix->n_slots; c.n_units = ix->n_units; c.slot_bytes = ix->slot_bytes; c.record_mode = ix->record_mode;
   c.ring = ix->ring_d; c.ring_mask = ix->ring_cap - 1; c.ring_shift = ilog2(ix->ring_cap);
   c.ring_dev = ix->ring_copy; c.host_ctl = ix->hctl_d;
   c.fdone = ix->fdone_d; c.host_pages = ix->pages_dev;
@@ -528,7 +549,7 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   // with every page resident one warp carries one query at a time, so no more than there are
   // queries per SM (fewer idle warps polling the queues), within 8..24
   u32 auto_warps = 16u;
-  if (ix->n_slots >= ix->n_pages) {
+  if (ix->n_slots >= ix->n_units) {
     auto_warps = (nq + (u32)ix->n_sms - 1) / (u32)ix->n_sms;
     auto_warps = auto_warps < 8u ? 8u : (auto_warps > 24u ? 24u : auto_warps);
   }
@@ -637,6 +658,7 @@ int gorio_stats(gorio_index *ix, gorio_stats_t *out) {
   out->proxy_iters = ix->host_iters; out->proxy_outstanding_sum = ix->host_out_sum;
   out->warp_ns_arrivals = h.stats[S_T_ARR]; out->warp_ns_queries = h.stats[S_T_RUN]; out->warp_ns_idle = h.stats[S_T_IDLE];
   out->arrivals_consumed = h.stats[S_N_ARR]; out->warp_ns_copies = h.stats[S_T_CPY]; out->stash_hits = h.stats[S_STASH];
+  out->fetched_bytes = ix->host_fetched_bytes;
   return GORIO_OK;
 }
 
@@ -644,6 +666,7 @@ int gorio_stats_reset(gorio_index *ix) {
   if (!ix) return GORIO_ERR_INVALID_ARG;
   CK(cudaSetDevice(ix->dev));
   CK(cudaMemset((u8 *)ix->ctl + offsetof(Ctl, stats), 0, sizeof(((Ctl *)0)->stats)));
+  ix->host_fetched_bytes = 0;
   ix->host_fetched = ix->host_max_out = ix->host_batches = ix->host_search_ns = 0;
   ix->host_service_ns = ix->host_ack_wait = ix->host_window_full = ix->host_ring_empty = ix->host_iters = ix->host_out_sum = 0;
   return GORIO_OK;

@@ -84,12 +84,16 @@ struct Ctx {
   const u8 *pq_codes;
   // page cache
   u8 *slot_data;   // n_slots * 4096
-  u64 *ptab;       // [n_pages] page words: state, slot, waiter-list head or generation
+  u64 *ptab;       // [n_units] page words: state, slot, waiter-list head or generation
   u64 *smeta;      // [n_slots] slot words: page, generation, reference bit
   u32 *parts;      // [n_slots] waiter-chain segments still being served
   u32 *filled;     // [n_slots] generation whose bytes the copier has stored into the slot
   CacheShared *cs; // clock hand and bump pointer
   u32 n_slots;
+  // cache unit: a 4 KB page (unit = node / npp, slot_bytes = 4096), or with selective
+  // materialisation one node record (unit = node; a slot holds the 16-byte-aligned span of the
+  // page that covers the record, so the record starts (offset in page) & 15 bytes into it)
+  u32 n_units, slot_bytes, record_mode;
   // miss ring: host-mapped, written by the GPU, consumed by the proxy
   u64 *ring;
   u32 ring_mask, ring_shift;

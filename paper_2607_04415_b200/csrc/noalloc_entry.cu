@@ -110,7 +110,7 @@ extern "C" int gorio_search_resident_noalloc(const gorio_index_desc *d, const vo
   c.n_nodes = (u32)d->n_nodes; c.dim = d->dim; c.dtype = d->dtype; c.R = R; c.npp = d->nodes_per_page;
   c.node_bytes = (u32)nb; c.vec_bytes = d->dim * esz; c.entry = d->entry_id; c.n_pages = (u32)n_pages;
   c.slot_data = (u8 *)const_cast<void *>(pages_dev);      // every page is resident: slot p holds page p
-  c.n_slots = (u32)n_pages;
+  c.n_slots = (u32)n_pages; c.n_units = (u32)n_pages; c.slot_bytes = kPageBytes; c.record_mode = 0;
   c.ctl = cv.take<Ctl>(1);
   c.cs = cv.take<CacheShared>(1);
   c.ptab = cv.take<u64>(n_pages); c.smeta = cv.take<u64>(n_pages);

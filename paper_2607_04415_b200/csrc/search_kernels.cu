@@ -151,6 +151,17 @@ __device__ __forceinline__ u64 mk_sm(u32 page, u32 gen, u32 ref) { return ((u64)
 __device__ __forceinline__ u32 sm_page(u64 m) { return (u32)(m >> 32); }
 __device__ __forceinline__ u32 sm_gen(u64 m) { return (u32)(m >> 1) & 0x7FFFFFFFu; }
 
+// The cache unit that holds `node` (a page, or with selective materialisation the node's own
+// record), and where the node's record starts inside the slot that holds that unit.
+__device__ __forceinline__ u32 unit_of(const Ctx &c, u32 node) { return c.record_mode ? node : node / c.npp; }
+__device__ __forceinline__ u32 rec_off(const Ctx &c, u32 node) {
+  const u32 off = (node % c.npp) * c.node_bytes;
+  return c.record_mode ? (off & 15u) : off;
+}
+__device__ __forceinline__ const u8 *rec_ptr(const Ctx &c, u32 slot, u32 node) {
+  return c.slot_data + (u64)slot * c.slot_bytes + rec_off(c, node);
+}
+
 struct LaneStats { u32 hit, missed, joins, evict, retry, posted; };
 
 // Post a request descriptor: one 64-bit word [page:32][slot:24][lap:8] in host-mapped memory.
@@ -183,7 +194,7 @@ __device__ u32 alloc_slot(const Ctx &c, u32 hint, LaneStats &st) {
     const u32 s = use_hint ? hint : atomicAdd(&c.cs->hand, 1u) % c.n_slots;
     const u64 m = ld_u64(c.smeta + s);
     const u32 pg = sm_page(m);
-    if (pg >= c.n_pages) continue;                       // slot handed out but not yet labelled
+    if (pg >= c.n_units) continue;                       // slot handed out but not yet labelled
     const u64 w = ld_u64(c.ptab + pg);
     if (pw_state(w) != P_RESIDENT || pw_slot(w) != s) continue;
     if ((m & 1ull) && !use_hint) {                       // referenced: second chance
@@ -298,7 +309,7 @@ __device__ void consume_item(const Ctx &c, u32 qs, u32 j, u32 slot, u32 lane) {
   const QHdr *h = c.hdr + qs;
   const u32 phase = ld_u32(&h->phase), qid = ld_u32(&h->qid);
   const u32 node = ld_u32(c.items + (u64)qs * c.WR + j);
-  const u8 *rec = c.slot_data + (u64)slot * kPageBytes + (node % c.npp) * c.node_bytes;
+  const u8 *rec = rec_ptr(c, slot, node);
   if (phase == PH_EVAL) {
     u32 d = warp_dist(c, rec, qid, lane);
     const u64 key = mk_key(d, node);
@@ -372,9 +383,9 @@ __device__ __forceinline__ u32 score_group128(const Ctx &c, u32 eval_mask, u32 q
       src[r] = valid[r] ? sel : 0u;
       const u32 s_qid = __shfl_sync(0xffffffffu, qid, src[r]), s_node = __shfl_sync(0xffffffffu, node, src[r]);
       const u32 s_slot = __shfl_sync(0xffffffffu, slot, src[r]);
-      const u32 off = (s_node % c.npp) * c.node_bytes;
+      const u32 off = rec_off(c, s_node);
       sw[r] = (off & 15u) >> 2;
-      const u8 *base = c.slot_data + (u64)s_slot * kPageBytes + (off & ~15u);
+      const u8 *base = c.slot_data + (u64)s_slot * c.slot_bytes + (off & ~15u);
       const u8 *q = (const u8 *)c.queries + (u64)s_qid * c.vec_bytes;
 #pragma unroll
       for (int k = 0; k < CH; ++k) {
@@ -461,7 +472,7 @@ __device__ __noinline__ void consume_group(const Ctx &c, u32 mask, u32 qs, u32 j
       if (g < ng) {
         const u32 s_qid = __shfl_sync(0xffffffffu, qid, src[g]), s_node = __shfl_sync(0xffffffffu, node, src[g]);
         const u32 s_slot = __shfl_sync(0xffffffffu, slot, src[g]);
-        const u32 *rec = (const u32 *)(c.slot_data + (u64)s_slot * kPageBytes + (s_node % c.npp) * c.node_bytes);
+        const u32 *rec = (const u32 *)rec_ptr(c, s_slot, s_node);
         const u32 *q = (const u32 *)((const u8 *)c.queries + (u64)s_qid * c.vec_bytes);
 #pragma unroll
         for (int w = 0; w < 3; ++w) {
@@ -506,7 +517,7 @@ __device__ __noinline__ void consume_group(const Ctx &c, u32 mask, u32 qs, u32 j
     u32 busy = 0;
     if (lane == 0) busy = atomicExch(tag, kStashBusy) == kStashBusy ? 1u : 0u;
     if (!__shfl_sync(0xffffffffu, busy, 0)) {
-      const u32 *adj = (const u32 *)(c.slot_data + (u64)s_slot * kPageBytes + (s_node % c.npp) * c.node_bytes + c.vec_bytes);
+      const u32 *adj = (const u32 *)(rec_ptr(c, s_slot, s_node) + c.vec_bytes);
       u32 *dst = c.stash + ((u64)s_qs * c.stash_cap + e) * (c.R + 1u);
       for (u32 i = lane; i < c.R + 1u; i += 32) st_u32(dst + i, __ldcg(adj + i));
       __syncwarp();
@@ -578,7 +589,7 @@ __device__ void consume_arrival(const Ctx &c, u32 v, u32 lane) {
     const u32 g = v & ~kContFlag;
     if (g >= c.n_qslots * c.WR) { if (lane == 0) raise(c, 8, 0x74, g); return; }
     const u32 node = uld(c.items + g);
-    const u32 page = node / c.npp;
+    const u32 page = unit_of(c, node);
     u64 w = ld_u64(c.ptab + page);
     w = __shfl_sync(0xffffffffu, w, 0);
     if (pw_state(w) != P_ARRIVED) { if (lane == 0) raise(c, 8, 0x75, g, page, (u32)(w >> 32)); return; }
@@ -590,7 +601,7 @@ __device__ void consume_arrival(const Ctx &c, u32 v, u32 lane) {
   u64 m = ld_u64(c.smeta + slot);
   m = __shfl_sync(0xffffffffu, m, 0);
   const u32 page = sm_page(m), gen = sm_gen(m);
-  if (page >= c.n_pages) { if (lane == 0) raise(c, 8, 0x76, slot, page); return; }
+  if (page >= c.n_units) { if (lane == 0) raise(c, 8, 0x76, slot, page); return; }
   u32 head = 0, bad = 0;
   if (lane == 0) {
     // acquire the copier's stores into the slot (normally long done: the completion was
@@ -657,14 +668,15 @@ __device__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
   for (u32 base = 0; base < n; base += 32) {
     const u32 j = base + lane;
     bool pending = j < n;
-    u32 node = 0, page = kInvalidId;
+    u32 node = 0, page = kInvalidId;      // page: the cache unit looked up (see unit_of)
     if (pending) {
       node = ld_u32(items + j);
-      page = node / c.npp;
-      if (count_pages) {
-        u32 r = set_insert(pset, c.pset_cap, page);
+      page = unit_of(c, node);
+      if (count_pages) {                  // distinct index pages, whatever the cache's unit
+        const u32 ipage = node / c.npp;
+        u32 r = set_insert(pset, c.pset_cap, ipage);
         if (r == 1) new_pages++;
-        else if (r == 2) raise(c, 6, 0x81, qs, page);
+        else if (r == 2) raise(c, 6, 0x81, qs, ipage);
       }
     }
     if (c.stash_cap && phase == PH_EXPAND && c.pq_m == 0) {
@@ -1204,12 +1216,22 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut, u32 &lut_qid
 __device__ void copy_page(const Ctx &c, u32 idx, u32 lane) {
   const u64 cmd = __shfl_sync(0xffffffffu, ld_u64(c.ring_dev + (idx & c.ring_mask)), 0);
   const u32 page = (u32)(cmd >> 32), slot = (u32)(cmd >> 8) & 0xFFFFFFu;
-  if (page >= c.n_pages || slot >= c.n_slots) { if (lane == 0) raise(c, 8, 0xC1, idx, page, slot); return; }
-  const uint4 *src = (const uint4 *)(c.host_pages + (u64)page * kPageBytes);
-  uint4 *dst = (uint4 *)(c.slot_data + (u64)slot * kPageBytes);
+  if (page >= c.n_units || slot >= c.n_slots) { if (lane == 0) raise(c, 8, 0xC1, idx, page, slot); return; }
+  // what to pull: the whole page, or (selective materialisation, Section 7.2) only the
+  // 16-byte-aligned span of its page that covers the wanted record
+  const uint4 *src;
+  u32 chunks = kPageBytes / 16u;
+  if (c.record_mode) {
+    const u32 off = (page % c.npp) * c.node_bytes;
+    src = (const uint4 *)(c.host_pages + (u64)(page / c.npp) * kPageBytes + (off & ~15u));
+    chunks = ((off & 15u) + c.node_bytes + 15u) >> 4;
+  } else {
+    src = (const uint4 *)(c.host_pages + (u64)page * kPageBytes);
+  }
+  uint4 *dst = (uint4 *)(c.slot_data + (u64)slot * c.slot_bytes);
   uint4 v[8];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) v[i] = __ldcs(src + i * 32 + lane);
+  for (int i = 0; i < 8; ++i) v[i] = (u32)i * 32u + lane < chunks ? __ldcs(src + i * 32 + lane) : make_uint4(0, 0, 0, 0);
   // The acknowledgement carries a checksum of the page above the lap tag (the host looks at the
   // tag only): a value that really depends on every loaded word, so the store cannot issue
   // before the page's bytes have arrived.
@@ -1219,7 +1241,7 @@ __device__ void copy_page(const Ctx &c, u32 idx, u32 lane) {
   sum = __reduce_xor_sync(0xffffffffu, sum);
   if (lane == 0) st_sys_u32(c.fdone + (idx & c.ring_mask), ((u32)cmd & 0xFFu) | (sum << 8));
 #pragma unroll
-  for (int i = 0; i < 8; ++i) __stcg(dst + i * 32 + lane, v[i]);
+  for (int i = 0; i < 8; ++i) if ((u32)i * 32u + lane < chunks) __stcg(dst + i * 32 + lane, v[i]);
   __syncwarp();          // orders every lane's stores before lane 0's release below
   if (lane == 0) {
     const u32 gen = sm_gen(ld_u64(c.smeta + slot));
@@ -1234,14 +1256,14 @@ __device__ void census(const Ctx &c, u32 lane) {
   for (u32 s = lane; s < c.n_slots; s += 32) {
     const u64 m = ld_u64(c.smeta + s);
     const u32 pg = sm_page(m);
-    if (pg >= c.n_pages) { cnt[0]++; continue; }
+    if (pg >= c.n_units) { cnt[0]++; continue; }
     const u64 w = ld_u64(c.ptab + pg);
     if (pw_slot(w) != s || pw_state(w) < P_FILLING) { cnt[1]++; continue; }   // slot between owners
     if (pw_state(w) == P_FILLING) cnt[2]++;
     else if (pw_state(w) == P_ARRIVED) cnt[3]++;
     else if (m & 1ull) cnt[4]++; else cnt[5]++;
   }
-  for (u32 p = lane; p < c.n_pages; p += 32) {
+  for (u32 p = lane; p < c.n_units; p += 32) {
     const u32 st = pw_state(ld_u64(c.ptab + p));
     if (st == P_WANTED) cnt[6]++;
   }
@@ -1387,7 +1409,7 @@ __global__ void init_kernel(const Ctx c) {
 // there by the host before this kernel) and are RESIDENT.
 __global__ void cache_reset_kernel(const Ctx c, u32 preloaded) {
   const u32 tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
-  for (u32 p = tid; p < c.n_pages; p += nth) c.ptab[p] = p < preloaded ? mk_pw(P_RESIDENT, p, 1) : kAbsentWord;
+  for (u32 p = tid; p < c.n_units; p += nth) c.ptab[p] = p < preloaded ? mk_pw(P_RESIDENT, p, 1) : kAbsentWord;
   for (u32 s = tid; s < c.n_slots; s += nth) {
     c.smeta[s] = s < preloaded ? mk_sm(s, 1, 1) : mk_sm(kInvalidId, 0, 0);
     c.parts[s] = 0;
