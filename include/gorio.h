@@ -117,7 +117,8 @@ enum { GORIO_GRAN_PAGE = 0, GORIO_GRAN_RECORD = 1 };
  *   max_inflight     query slots resident at once (pending/running queries); default 16384.
  *   visited_capacity per-query exact visited-set entries (power of two), default 32768;
  *                    a query that scores more nodes fails with GORIO_ERR_CAPACITY.
- *   warps_per_block / blocks_per_sm  launch geometry of the persistent kernel (<= 24 warps).
+ *   warps_per_block / blocks_per_sm  launch geometry of the persistent kernel (<= 24 warps; with
+ *                    PQ navigation at most 12, fewer if the per-warp tables do not fit).
  *   stash_entries    per-query adjacency stash (exact navigation): entries of a direct-mapped
  *                    table that keeps a scored node's neighbour list so that expanding it later
  *                    needs no page; 0 = default 1024, 1 = off, else a power of two >= 64.

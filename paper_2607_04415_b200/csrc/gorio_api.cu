@@ -542,6 +542,7 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   if (c.max_in_flight < ix->cfg.max_outstanding) c.max_in_flight = ix->cfg.max_outstanding;
   c.vec128 = (ix->vec_bytes % 16 == 0 && ix->vec_bytes <= 384 && ((uintptr_t)queries_dev & 15) == 0) ? 1u : 0u;
   { const char *e = std::getenv("GORIO_CENSUS_MS"); c.census_ns = e ? (u64)std::atof(e) * 1000000ull : 0; }
+  c.prof = std::getenv("GORIO_PROFILE") ? 1u : 0u;
 
   // launch geometry: one block per SM by default
   const bool pq = d.pq_m != 0;
@@ -554,7 +555,11 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
     auto_warps = auto_warps < 8u ? 8u : (auto_warps > 24u ? 24u : auto_warps);
   }
   u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 10u : auto_warps);
-  if (pq) { u32 lim = (220u * 1024u) / (d.pq_m * kPqLutWords * 4u); if (warps > lim) warps = lim; }
+  if (pq) {      // one table per warp in shared memory; the PQ kernel is built for at most 12 warps
+    u32 lim = (220u * 1024u) / (d.pq_m * kPqLutWords * 4u);
+    if (lim > 12u) lim = 12u;
+    if (warps > lim) warps = lim;
+  }
   if (warps < 2) return fail(ix, GORIO_ERR_INVALID_ARG, "search: need at least 2 warps per block (the poller and a worker)");
   int occ = 0;
   CK(search_occupancy(d.pq_m, warps, &occ));
@@ -599,6 +604,14 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
                  "pages WANTED %u | queries awaiting %u (items %u) | queues want %d arr %d run %d | done %u posted %u\n",
                  h.census[0], h.census[1], h.census[2], h.census[3], h.census[4], h.census[5], h.census[6], h.census[7],
                  h.census[8], (int)h.census[9], (int)h.census[10], (int)h.census[11], h.census[12], h.census[13]);
+  if (c.prof) {
+    const char *names[] = {"merge", "issue_eval", "issue_expand", "collect", "pool", "lut", "adc", "finish", "recycle",
+                           "(issue: setup", "lookup", "consume", "tail)"};
+    std::fprintf(stderr, "[gorio profile] warp ms per query step (cumulative since stats_reset):");
+    for (int i = 0; i < 13; ++i) std::fprintf(stderr, " %s %.1f", names[i], h.stats[S_P_MERGE + i] / 1e6);
+    std::fprintf(stderr, " | arrivals %.1f copies %.1f queries %.1f idle %.1f\n", h.stats[S_T_ARR] / 1e6, h.stats[S_T_CPY] / 1e6,
+                 h.stats[S_T_RUN] / 1e6, h.stats[S_T_IDLE] / 1e6);
+  }
   if (ix->px_error.load()) return fail(ix, GORIO_ERR_INTERNAL, "proxy: descriptor out of range");
   if (h.status != 0 || h.stop != 1) {
     char buf[640];

@@ -73,7 +73,10 @@ struct Ctl {
 };
 
 enum StatIdx { S_HIT = 0, S_MISSED, S_JOINS, S_EVICT, S_RETRY, S_DONE, S_NEVAL, S_NEXPAND,
-               S_SUMDEG, S_NITER, S_RESUMES, S_POSTED, S_T_ARR, S_T_RUN, S_T_IDLE, S_N_ARR, S_T_CPY, S_STASH };
+               S_SUMDEG, S_NITER, S_RESUMES, S_POSTED, S_T_ARR, S_T_RUN, S_T_IDLE, S_N_ARR, S_T_CPY, S_STASH,
+               // debug profile (Ctx::prof): warp time per query phase step
+               S_P_MERGE, S_P_ISSUE_EVAL, S_P_ISSUE_EXP, S_P_COLLECT, S_P_POOL, S_P_LUT, S_P_ADC, S_P_FINISH, S_P_RECYCLE,
+               S_I_SETUP, S_I_LOOKUP, S_I_CONSUME, S_I_TAIL };   // inside issue_batch
 
 // Everything the persistent kernel needs, passed by value.
 struct Ctx {
@@ -132,6 +135,7 @@ struct Ctx {
   u32 max_in_flight; // cap on posted-but-not-arrived requests
   u32 vec128;      // 1: vectors are whole 16-byte chunks (<= 24) and query rows are 16-byte aligned
   u32 blocking;    // 1: a warp waits in place for its query's pages instead of yielding
+  u32 prof;        // debug: 1 = account warp time per query phase step in stats[S_P_*]
 };
 
 // launchers implemented in search_kernels.cu

@@ -179,10 +179,20 @@ __device__ __forceinline__ void post_request(const Ctx &c, u32 page, u32 slot) {
   st_sys_u64(c.ring + (idx & c.ring_mask), e);
 }
 
+// Requests posted and not yet arrived are kept near a small multiple of the proxy's window:
+// anything more would only queue in the ring while holding a slot that could keep a resident
+// page instead (with the whole cache in flight it is a buffer pool, not a cache).
+__device__ __forceinline__ bool may_post(const Ctx &c) { return (int)ld_u32((const u32 *)&c.cs->in_flight) < (int)c.max_in_flight; }
+
 // Get a slot for a new page: never-used slots first, then the clock (second chance for
 // referenced pages); `hint` (a slot the caller has just made evictable) is taken if a short
-// sweep finds nothing.  Returns kNil when every slot examined is in flight.
-__device__ u32 alloc_slot(const Ctx &c, u32 hint, LaneStats &st) {
+// sweep finds nothing.  Returns kNil when every slot examined is in flight; otherwise `prev_gen`
+// is the generation of the slot's previous fill.  (The backlog gate, may_post, stays with the
+// callers: checking it again here made serve_want put pages it had already popped back at the
+// tail of the want queue, the queue stopped being first-in first-out, requests were posted
+// with far fewer waiters each, and config 3 fetched 9.3 M pages instead of 3.7 M.)
+__device__ u32 alloc_slot(const Ctx &c, u32 hint, LaneStats &st, u32 &prev_gen) {
+  prev_gen = 0;
   if (ld_u32(&c.cs->bump) < c.n_slots) {
     u32 b = atomicAdd(&c.cs->bump, 1u);
     if (b < c.n_slots) return b;
@@ -201,41 +211,42 @@ __device__ u32 alloc_slot(const Ctx &c, u32 hint, LaneStats &st) {
       atomicCAS((unsigned long long *)(c.smeta + s), m, m & ~1ull);
       continue;
     }
-    if (atomicCAS((unsigned long long *)(c.ptab + pg), w, kAbsentWord) == w) { st.evict++; return s; }
+    if (atomicCAS((unsigned long long *)(c.ptab + pg), w, kAbsentWord) == w) {
+      st.evict++;
+      prev_gen = sm_gen(m);
+      return s;
+    }
   }
   return kNil;
 }
 
 // The page is WANTED and `slot` is exclusively ours: label the slot, move the page to
 // FILLING (keeping whatever waiters have queued up meanwhile) and post the descriptor.
-__device__ void assign_and_post(const Ctx &c, u32 page, u32 slot, LaneStats &st) {
-  const u32 gen = sm_gen(ld_u64(c.smeta + slot)) + 1u;
-  st_u64(c.smeta + slot, mk_sm(page, gen, 0));
+// `expect` is what the caller believes the page word to be (0 = not known).
+__device__ void assign_and_post(const Ctx &c, u32 page, u32 slot, u32 prev_gen, u64 expect, LaneStats &st) {
+  st_u64(c.smeta + slot, mk_sm(page, prev_gen + 1u, 0));
   // (no fence needed here: a clock sweep that sees the new label with the old page word, or
   // the reverse, finds state != RESIDENT or a slot mismatch and moves on; everyone else
   // learns of the slot through the descriptor, which is fenced in post_request)
+  u64 w = expect ? expect : ld_u64(c.ptab + page);
   for (u32 spins = 0;; ++spins) {
-    const u64 w = ld_u64(c.ptab + page);
     if (pw_state(w) != P_WANTED || spins > kSpinLimit) { raise(c, 8, 0x41, page, (u32)(w >> 32), spins); return; }
-    if (atomicCAS((unsigned long long *)(c.ptab + page), w, mk_pw(P_FILLING, slot, pw_low(w))) == w) break;
+    const u64 old = atomicCAS((unsigned long long *)(c.ptab + page), w, mk_pw(P_FILLING, slot, pw_low(w)));
+    if (old == w) break;
+    w = old;
   }
   post_request(c, page, slot);
   st.posted++;
 }
 
 // Serve one page from the want queue if a slot can be had (one lane).
-// Requests posted and not yet arrived are kept near a small multiple of the proxy's window:
-// anything more would only queue in the ring while holding a slot that could keep a resident
-// page instead (with the whole cache in flight it is a buffer pool, not a cache).
-__device__ __forceinline__ bool may_post(const Ctx &c) { return (int)ld_u32((const u32 *)&c.cs->in_flight) < (int)c.max_in_flight; }
-
 __device__ void serve_want(const Ctx &c, u32 hint, LaneStats &st) {
-  u32 page;
+  u32 page, prev_gen = 0;
   if (!may_post(c)) return;
   if (!q_pop(c, c.want, page)) return;
-  const u32 slot = alloc_slot(c, hint, st);
+  const u32 slot = alloc_slot(c, hint, st, prev_gen);
   if (slot == kNil) { q_push(c, c.want, page); return; }
-  assign_and_post(c, page, slot, st);
+  assign_and_post(c, page, slot, prev_gen, 0, st);
 }
 
 // Lookup / miss generation for one item by one lane.  g is the item's waiter record.
@@ -251,11 +262,23 @@ __device__ u32 page_lookup(const Ctx &c, u32 page, u32 g, u32 &slot, u32 &gen, L
     st_u32(c.wrec + g, s == P_ABSENT ? kNil : pw_low(w));
     __threadfence();
     if (s == P_ABSENT) {
-      if (atomicCAS((unsigned long long *)pw, w, mk_pw(P_WANTED, 0, g)) != w) continue;
+      const u64 wanted = mk_pw(P_WANTED, 0, g);
+      if (atomicCAS((unsigned long long *)pw, w, wanted) != w) continue;
       st.missed++;
-      const u32 sl = may_post(c) ? alloc_slot(c, kNil, st) : kNil;   // first requester: find the page a slot
-      if (sl != kNil) assign_and_post(c, page, sl, st);
-      else q_push(c, c.want, page);
+      // First requester: find the page a slot -- but never ahead of pages that already wait for
+      // one.  Requests leave in the order in which their pages were first wanted, so each has
+      // gathered as many waiters as it can by the time it is posted; letting new pages jump the
+      // queue whenever the backlog had room cost 16 % more fetches on config 3.
+      const bool room = may_post(c);
+      const bool queued = (int)ld_u32((const u32 *)c.want.count) > 0;
+      u32 prev_gen = 0;
+      const u32 sl = (room && !queued) ? alloc_slot(c, kNil, st, prev_gen) : kNil;
+      if (sl != kNil) {
+        assign_and_post(c, page, sl, prev_gen, wanted, st);
+      } else {
+        q_push(c, c.want, page);
+        if (room) serve_want(c, kNil, st);      // the oldest waiting page takes the opening
+      }
       return LK_WAIT;
     }
     if (atomicCAS((unsigned long long *)pw, w, (w & 0xFFFFFFFF00000000ull) | g) != w) continue;
@@ -644,6 +667,14 @@ __device__ u32 set_insert(u32 *tab, u32 cap, u32 v) {
   return 2;
 }
 
+// Debug profile: charge the time since `t` to stats[idx] and restart the clock.
+__device__ __forceinline__ void phase_mark(const Ctx &c, u64 &t, u32 idx, u32 lane) {
+  if (!c.prof) return;
+  const u64 now = globaltimer();
+  if (lane == 0) atomicAdd((unsigned long long *)&c.ctl->stats[idx], now - t);
+  t = now;
+}
+
 // ------------------------------------------------------------------------------------------
 // issue a batch of page items for query slot qs
 // ------------------------------------------------------------------------------------------
@@ -664,6 +695,7 @@ __device__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
   u32 *pset = c.pset + (u64)qs * c.pset_cap;
   LaneStats st = {0, 0, 0, 0, 0, 0};
   u32 n_done = 0, new_pages = 0, n_stash = 0;
+  u64 tq = c.prof ? globaltimer() : 0;
 
   for (u32 base = 0; base < n; base += 32) {
     const u32 j = base + lane;
@@ -702,10 +734,12 @@ __device__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
         }
       }
     }
+    phase_mark(c, tq, S_I_SETUP, lane);
     for (u32 round = 0; __any_sync(0xffffffffu, pending); ++round) {
       u32 code = LK_NONE, slot = 0, gen = 0;
       if (pending) code = page_lookup(c, page, qs * c.WR + j, slot, gen, st);
       __syncwarp();
+      phase_mark(c, tq, S_I_LOOKUP, lane);
       if (code == LK_WAIT) pending = false;
       const u32 hits = __ballot_sync(0xffffffffu, code == LK_HIT);
       if (hits) consume_group(c, hits, qs, j, slot, lane);
@@ -725,6 +759,7 @@ __device__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
           }
         }
       }
+      phase_mark(c, tq, S_I_CONSUME, lane);
       if (round > 1024) { if (lane == 0) raise(c, 8, 0x84, qs, base); break; }
       if (warp_stopped(c)) break;
     }
@@ -744,18 +779,18 @@ __device__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
     st.posted += __shfl_xor_sync(0xffffffffu, st.posted, o);
   }
   u32 complete = 0;
+  if (lane == 0 && new_pages) atomicAdd(&h->pages_distinct, new_pages);   // only this warp touches it while it holds the guard
   __threadfence();
   __syncwarp();
   if (lane == 0) {
-    stat_add(c, S_HIT, st.hit); stat_add(c, S_MISSED, st.missed); stat_add(c, S_JOINS, st.joins);
-    stat_add(c, S_EVICT, st.evict); stat_add(c, S_RETRY, st.retry); stat_add(c, S_POSTED, st.posted);
-    stat_add(c, S_STASH, n_stash);
-    if (new_pages) st_u32(&h->pages_distinct, ld_u32(&h->pages_distinct) + new_pages);
-    __threadfence();
     const u32 old = atomicSub(&h->awaiting, n_done + 1u);       // inline hits and the guard
     if (old == n_done + 1u) complete = 1;
     else if (old < n_done + 1u) raise(c, 8, 0x82, qs, old, n_done);
+    stat_add(c, S_HIT, st.hit); stat_add(c, S_MISSED, st.missed); stat_add(c, S_JOINS, st.joins);
+    stat_add(c, S_EVICT, st.evict); stat_add(c, S_RETRY, st.retry); stat_add(c, S_POSTED, st.posted);
+    stat_add(c, S_STASH, n_stash);
   }
+  phase_mark(c, tq, S_I_TAIL, lane);
   return __shfl_sync(0xffffffffu, complete, 0) != 0u;
 }
 
@@ -1001,30 +1036,87 @@ __device__ __forceinline__ u32 lut_get(const u16 *lo, const u32 *hi, u32 e) {
   return (u32)lo[e] | (((hi[e >> 3] >> ((e & 7u) * 4u)) & 15u) << 16);
 }
 
-__device__ void build_lut(const Ctx &c, u32 qid, u32 *lut, u32 lane) {
-  const u8 *q = (const u8 *)c.queries + (u64)qid * c.vec_bytes;
-  const u32 wsub = c.pq_dsub >> 2;
-  const u32 total = c.pq_m * kPqKsub;
-  u16 *lo = (u16 *)lut;
+// Building the table reads the whole codebook (pq_m x 256 centroids, L2 resident).  A query that
+// is resumed on another warp rebuilds it, so the loads are issued in batches before any result
+// is needed: one load at a time costs an L2 round trip per entry (86 us per table measured).
+//
+// dsub == 4 (one word per centroid) with a 16-byte-aligned codebook: a lane takes four
+// consecutive entries per 16-byte load, eight loads in flight.
+__device__ void build_lut_w1(const Ctx &c, const u8 *q, u32 *lut, u32 lane) {
+  const u32 quads = c.pq_m * (kPqKsub / 4);
+  const uint4 *cent = (const uint4 *)c.pq_cent;
+  uint2 *lo2 = (uint2 *)lut;
   u32 *hi = lut + c.pq_m * (kPqKsub / 2);
-  for (u32 e = lane; e < total; e += 32) {            // total is a multiple of 32: no lane idles
-    const u32 m = e >> 8;
-    const u32 *cw = (const u32 *)(c.pq_cent + (u64)e * c.pq_dsub);
-    const u32 *qw = (const u32 *)(q + m * c.pq_dsub);
-    u32 s = 0;
-    for (u32 w = 0; w < wsub; ++w) {
-      u32 d = __vabsdiffu4(__ldg(cw + w), __ldg(qw + w));
-      s = __dp4a(d, d, s);
+  for (u32 g0 = lane; g0 < quads; g0 += 32u * 8u) {
+    uint4 cw[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const u32 g = g0 + 32u * (u32)k;
+      cw[k] = g < quads ? __ldg(cent + g) : make_uint4(0, 0, 0, 0);
     }
-    lo[e] = (u16)s;
-    // eight consecutive entries (lanes 8k..8k+7) share one word of high nibbles
-    u32 nib = ((s >> 16) & 15u) << ((lane & 7u) * 4u);
-    nib |= __shfl_xor_sync(0xffffffffu, nib, 1);
-    nib |= __shfl_xor_sync(0xffffffffu, nib, 2);
-    nib |= __shfl_xor_sync(0xffffffffu, nib, 4);
-    if ((lane & 7u) == 0) hi[e >> 3] = nib;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const u32 g = g0 + 32u * (u32)k;
+      const bool in = g < quads;                         // the same for a lane and its partner: quads is even
+      const u32 qw = in ? __ldg((const u32 *)q + (g >> 6)) : 0u;     // 64 groups of four per subspace
+      u32 d, s0, s1, s2, s3;
+      d = __vabsdiffu4(cw[k].x, qw); s0 = __dp4a(d, d, 0u);
+      d = __vabsdiffu4(cw[k].y, qw); s1 = __dp4a(d, d, 0u);
+      d = __vabsdiffu4(cw[k].z, qw); s2 = __dp4a(d, d, 0u);
+      d = __vabsdiffu4(cw[k].w, qw); s3 = __dp4a(d, d, 0u);
+      if (in) lo2[g] = make_uint2((s0 & 0xFFFFu) | (s1 << 16), (s2 & 0xFFFFu) | (s3 << 16));
+      // entries 4g..4g+3 are half of the high-nibble word g >> 1; the neighbouring lane holds the other half
+      const u32 nib = ((s0 >> 16) & 15u) | (((s1 >> 16) & 15u) << 4) | (((s2 >> 16) & 15u) << 8) | (((s3 >> 16) & 15u) << 12);
+      const u32 other = __shfl_xor_sync(0xffffffffu, nib, 1);
+      if (in && (lane & 1u) == 0u) hi[g >> 1] = nib | (other << 16);
+    }
   }
   __syncwarp();
+}
+
+template <int WSUB>
+__device__ void build_lut_gen(const Ctx &c, const u8 *q, u32 *lut, u32 lane) {
+  const u32 total = c.pq_m * kPqKsub;                  // a multiple of 256: no lane ever idles
+  u16 *lo = (u16 *)lut;
+  u32 *hi = lut + c.pq_m * (kPqKsub / 2);
+  for (u32 e0 = lane; e0 < total; e0 += 32u * 4u) {
+    u32 cw[4][WSUB];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const u32 *p = (const u32 *)(c.pq_cent + (u64)(e0 + 32u * (u32)u) * c.pq_dsub);
+#pragma unroll
+      for (int w = 0; w < WSUB; ++w) cw[u][w] = __ldg(p + w);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const u32 e = e0 + 32u * (u32)u;
+      const u32 *qw = (const u32 *)(q + (e >> 8) * c.pq_dsub);
+      u32 s = 0;
+#pragma unroll
+      for (int w = 0; w < WSUB; ++w) { const u32 d = __vabsdiffu4(cw[u][w], __ldg(qw + w)); s = __dp4a(d, d, s); }
+      lo[e] = (u16)s;
+      // eight consecutive entries (lanes 8k..8k+7) share one word of high nibbles
+      u32 nib = ((s >> 16) & 15u) << ((lane & 7u) * 4u);
+      nib |= __shfl_xor_sync(0xffffffffu, nib, 1);
+      nib |= __shfl_xor_sync(0xffffffffu, nib, 2);
+      nib |= __shfl_xor_sync(0xffffffffu, nib, 4);
+      if ((lane & 7u) == 0) hi[e >> 3] = nib;
+    }
+  }
+  __syncwarp();
+}
+
+__device__ __noinline__ void build_lut(const Ctx &c, u32 qid, u32 *lut, u32 lane) {
+  const u8 *q = (const u8 *)c.queries + (u64)qid * c.vec_bytes;
+  switch (c.pq_dsub >> 2) {
+    case 1:
+      if (((uintptr_t)c.pq_cent & 15u) == 0) build_lut_w1(c, q, lut, lane);
+      else build_lut_gen<1>(c, q, lut, lane);
+      break;
+    case 2: build_lut_gen<2>(c, q, lut, lane); break;
+    case 3: build_lut_gen<3>(c, q, lut, lane); break;
+    default: build_lut_gen<4>(c, q, lut, lane); break;
+  }
 }
 // One node per lane: the lane reads the node's code (pq_m bytes, 4 at a time) and sums pq_m
 // independent table entries from shared memory -- no cross-lane reduction, 32 nodes per pass.
@@ -1145,6 +1237,7 @@ __device__ __noinline__ bool wait_in_place(const Ctx &c, u32 qs, u32 lane) {
 template <bool PQ>
 __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut, u32 &lut_qid) {
   QHdr *h = c.hdr + qs;
+  u64 tp = c.prof ? globaltimer() : 0;
   for (u32 guard = 0; guard < 4u * c.max_iters + 64u; ++guard) {
     if (warp_stopped(c)) return;
     const u32 phase = uld(&h->phase);
@@ -1158,16 +1251,23 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut, u32 &lut_qid
       __syncwarp();
       if (PQ) {
         if (lut_qid != qid) { build_lut(c, qid, lut, lane); lut_qid = qid; }
+        phase_mark(c, tp, S_P_LUT, lane);
         if (lane == 0) st_u64(c.cand + (u64)qs * c.WR, mk_key(lane_adc(c, lut, c.entry), c.entry));
         __syncwarp();
       } else {
-        if (!issue_batch(c, qs, lane) && !(c.blocking && wait_in_place(c, qs, lane))) return;
+        const bool go = issue_batch(c, qs, lane);
+        phase_mark(c, tp, S_P_ISSUE_EVAL, lane);
+        if (!go && !(c.blocking && wait_in_place(c, qs, lane))) return;
       }
     } else if (phase == PH_EVAL) {
       const u32 nf = merge_select_dispatch(c, qs, lane);
+      phase_mark(c, tp, S_P_MERGE, lane);
       if (nf == 0) {
         finish_query(c, qs, lane);
-        if (!recycle_slot(c, qs, lane)) return;
+        phase_mark(c, tp, S_P_FINISH, lane);
+        const bool more = recycle_slot(c, qs, lane);
+        phase_mark(c, tp, S_P_RECYCLE, lane);
+        if (!more) return;
         guard = 0;
         continue;
       }
@@ -1178,14 +1278,21 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut, u32 &lut_qid
         if (it > c.max_iters) raise(c, 6, 0xA1, qs, it);
       }
       __syncwarp();
-      if (!issue_batch(c, qs, lane) && !(c.blocking && wait_in_place(c, qs, lane))) return;
+      {
+        const bool go = issue_batch(c, qs, lane);
+        phase_mark(c, tp, S_P_ISSUE_EXP, lane);
+        if (!go && !(c.blocking && wait_in_place(c, qs, lane))) return;
+      }
     } else {  // PH_EXPAND complete
       const u32 nf = uld(&h->n_items);
       const u32 nn = collect_neighbors(c, qs, lane);
+      phase_mark(c, tp, S_P_COLLECT, lane);
       if (PQ) {
         pool_merge_dispatch(c, qs, nf, false, lane);
+        phase_mark(c, tp, S_P_POOL, lane);
         const u32 qid = uld(&h->qid);
         if (lut_qid != qid) { build_lut(c, qid, lut, lane); lut_qid = qid; }
+        phase_mark(c, tp, S_P_LUT, lane);
         const u32 *items = c.items + (u64)qs * c.WR;
         for (u32 base = 0; base < nn; base += 32) {
           const u32 i = base + lane;
@@ -1195,11 +1302,14 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut, u32 &lut_qid
           }
         }
         __syncwarp();
+        phase_mark(c, tp, S_P_ADC, lane);
       }
       if (lane == 0) { st_u32(&h->n_items, nn); st_u32(&h->phase, PH_EVAL); }
       __syncwarp();
       if (!PQ && nn > 0) {
-        if (!issue_batch(c, qs, lane) && !(c.blocking && wait_in_place(c, qs, lane))) return;
+        const bool go = issue_batch(c, qs, lane);
+        phase_mark(c, tp, S_P_ISSUE_EVAL, lane);
+        if (!go && !(c.blocking && wait_in_place(c, qs, lane))) return;
       }
     }
   }
@@ -1220,7 +1330,7 @@ __device__ void copy_page(const Ctx &c, u32 idx, u32 lane) {
   // what to pull: the whole page, or (selective materialisation, Section 7.2) only the
   // 16-byte-aligned span of its page that covers the wanted record
   const uint4 *src;
-  u32 chunks = kPageBytes / 16u;
+  u32 chunks = kPageBytes / 16u;      // page granularity moves the whole 4 KB block, as a block device would
   if (c.record_mode) {
     const u32 off = (page % c.npp) * c.node_bytes;
     src = (const uint4 *)(c.host_pages + (u64)(page / c.npp) * kPageBytes + (off & ~15u));
@@ -1322,9 +1432,11 @@ __device__ bool warp_ticket(int *count, u32 *head, u32 &idx, u32 lane) {
   return __shfl_sync(0xffffffffu, ok, 0) != 0u;
 }
 
-// Register budget: at most 80 per thread, so that 24 warps (61,440 registers) fit on an SM.
+// Register budget: at most 80 per thread, so that 24 warps (61,440 registers) fit on an SM.  With
+// PQ navigation the per-warp table in shared memory allows 12 warps at most, so that variant is
+// built for 384 threads and may use twice the registers (no spills).
 template <bool PQ>
-__global__ void __launch_bounds__(768, 1) search_kernel(const Ctx c) {
+__global__ void __launch_bounds__(PQ ? 384 : 768, 1) search_kernel(const Ctx c) {
   extern __shared__ u32 smem_lut[];
   const u32 lane = lane_id(), warp = threadIdx.x >> 5;
   if (blockIdx.x == 0 && warp == 0) { poller(c, lane); return; }

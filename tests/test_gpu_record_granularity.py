@@ -62,6 +62,7 @@ def test_fewer_bytes_cross_the_link_than_at_page_granularity(gorio, cfg1):
     _assert_exact(page, ref)
     _assert_exact(rec, ref)
     assert page["stats"]["fetched_bytes"] == page["stats"]["pages_fetched"] * 4096
+    assert rec["stats"]["fetched_bytes"] == rec["stats"]["pages_fetched"] * _slot_bytes(w)
     assert rec["stats"]["fetched_bytes"] * 2 < page["stats"]["fetched_bytes"]
 
 
