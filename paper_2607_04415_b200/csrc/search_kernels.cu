@@ -253,10 +253,12 @@ __device__ void serve_want(const Ctx &c, u32 hint, LaneStats &st) {
 // Returns LK_HIT with (slot, generation) to be consumed and validated by the caller, or
 // LK_WAIT when the item now waits on the page (as first requester or as a joiner).
 enum LookupCode : u32 { LK_NONE = 0, LK_HIT = 1, LK_WAIT = 2 };
-__device__ u32 page_lookup(const Ctx &c, u32 page, u32 g, u32 &slot, u32 &gen, LaneStats &st) {
+// `first` is the page word as the caller last saw it (every decision below is re-checked by a
+// compare-and-swap or by the caller's validation, so a stale word only costs a retry).
+__device__ u32 page_lookup(const Ctx &c, u32 page, u32 g, u64 first, u32 &slot, u32 &gen, LaneStats &st) {
   u64 *pw = c.ptab + page;
   for (u32 tries = 0; tries < 4096; ++tries) {
-    const u64 w = ld_u64(pw);
+    const u64 w = tries ? ld_u64(pw) : first;
     const u32 s = pw_state(w);
     if (s == P_RESIDENT || s == P_ARRIVED) { slot = pw_slot(w); gen = pw_low(w); return LK_HIT; }
     st_u32(c.wrec + g, s == P_ABSENT ? kNil : pw_low(w));
@@ -468,16 +470,14 @@ __device__ __forceinline__ u32 score_group128(const Ctx &c, u32 eval_mask, u32 q
 // L2 round trips of different items overlap instead of adding up (the per-item version is
 // latency bound).  Adjacency copies (expansion items) and vectors longer than 96 words take
 // the one-at-a-time path.
-__device__ __noinline__ void consume_group(const Ctx &c, u32 mask, u32 qs, u32 j, u32 slot, u32 lane) {
+//
+// Lane i also holds its item's metadata: the query's phase and id, the node, and (exact
+// navigation with a stash) the list's worst key as of the last merge.
+template <bool PQ>
+__device__ __noinline__ void consume_group(const Ctx &c, u32 mask, u32 qs, u32 j, u32 slot, u32 phase, u32 qid,
+                                           u32 node, u64 worst, u32 lane) {
   const bool mine = (mask >> lane) & 1u;
-  u32 phase = 0, qid = 0, node = 0;
-  u64 worst = 0;
-  if (mine) {
-    const QHdr *h = c.hdr + qs;
-    phase = ld_u32(&h->phase); qid = ld_u32(&h->qid);
-    node = ld_u32(c.items + (u64)qs * c.WR + j);
-    if (c.stash_cap) worst = ld_u64((const u64 *)&h->worst_lo);
-  }
+  if (!mine) { phase = 0; qid = 0; node = 0; worst = 0; }
   const u32 words = c.vec_bytes >> 2;
   const u32 eval_mask = words <= 96u ? __ballot_sync(0xffffffffu, mine && phase == PH_EVAL) : 0u;
   u32 dist = 0;
@@ -547,8 +547,67 @@ __device__ __noinline__ void consume_group(const Ctx &c, u32 mask, u32 qs, u32 j
       if (lane == 0) { __threadfence(); st_u32(tag, s_node); }
     }
   }
+  // Expansion items: copy the node's adjacency list into the query's buffer (PQ navigation: also
+  // its exact distance into the rerank pool's staging entries), two items' loads in flight.
+  const u32 rest = mask & ~eval_mask;
+  const bool paired = words <= 96u && c.R + 1u <= 96u;
+  for (u32 m = paired ? rest : 0u; m;) {
+    u32 src[2], a[2][3], v[2][3], qw[2][3];
+    int ng = 0;
+#pragma unroll
+    for (int g = 0; g < 2; ++g) { src[g] = 0; if (m) { src[g] = __ffs(m) - 1; m &= m - 1; ng = g + 1; } }
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+      if (g < ng) {
+        const u32 s_node = __shfl_sync(0xffffffffu, node, src[g]), s_slot = __shfl_sync(0xffffffffu, slot, src[g]);
+        const u32 s_qid = __shfl_sync(0xffffffffu, qid, src[g]);
+        const u32 *rec = (const u32 *)rec_ptr(c, s_slot, s_node);
+        const u32 *adj = rec + words;                       // degree, then R ids
+        const u32 *q = (const u32 *)((const u8 *)c.queries + (u64)s_qid * c.vec_bytes);
+#pragma unroll
+        for (int k = 0; k < 3; ++k) {
+          const u32 idx = (u32)k * 32u + lane;
+          a[g][k] = idx <= c.R ? __ldcg(adj + idx) : 0u;
+          const bool in = PQ && idx < words;
+          v[g][k] = in ? __ldcg(rec + idx) : 0u;
+          qw[g][k] = in ? __ldg(q + idx) : 0u;
+        }
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+      if (g < ng) {
+        const u32 s_qs = __shfl_sync(0xffffffffu, qs, src[g]), s_j = __shfl_sync(0xffffffffu, j, src[g]);
+        const u32 s_node = __shfl_sync(0xffffffffu, node, src[g]);
+        u32 *dst = c.adj + ((u64)s_qs * c.W + s_j) * c.R;
+#pragma unroll
+        for (int k = 0; k < 3; ++k) {
+          const u32 idx = (u32)k * 32u + lane;
+          if (idx >= 1u && idx <= c.R) st_u32(dst + idx - 1u, a[g][k]);
+        }
+        if (lane == 0) st_u32(c.adjdeg + (u64)s_qs * c.W + s_j, a[g][0]);
+        if (PQ) {
+          u32 d;
+          if (c.dtype == 0) {
+            u32 acc = 0;
+#pragma unroll
+            for (int k = 0; k < 3; ++k) { const u32 x = __vabsdiffu4(v[g][k], qw[g][k]); acc = __dp4a(x, x, acc); }
+            d = __reduce_add_sync(0xffffffffu, acc);
+          } else {                                          // same order as warp_dist
+            float acc = 0.f;
+#pragma unroll
+            for (int k = 0; k < 3; ++k) { const float x = __uint_as_float(qw[g][k]) - __uint_as_float(v[g][k]); acc = fmaf(x, x, acc); }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            d = __float_as_uint(acc);
+          }
+          if (lane == 0) st_u64(c.pool + (u64)s_qs * (c.K + c.W) + c.K + s_j, mk_key(d, s_node));
+        }
+      }
+    }
+  }
   // everything else one at a time
-  for (u32 m = mask & ~eval_mask; m; m &= m - 1) {
+  for (u32 m = paired ? 0u : rest; m; m &= m - 1) {
     const u32 src = __ffs(m) - 1;
     consume_item(c, __shfl_sync(0xffffffffu, qs, src), __shfl_sync(0xffffffffu, j, src),
                  __shfl_sync(0xffffffffu, slot, src), lane);
@@ -576,6 +635,7 @@ __device__ void finish_arrival(const Ctx &c, u32 slot, u32 page, u32 gen, u32 la
 }
 
 // Consume the waiter chain starting at record g for the page held in `slot`.
+template <bool PQ>
 __device__ void consume_chain(const Ctx &c, u32 slot, u32 page, u32 gen, u32 g, u32 lane) {
   const u32 limit = c.n_qslots * c.WR;
   // chase up to a segment of next pointers first so that the remainder is handed off early
@@ -593,7 +653,15 @@ __device__ void consume_chain(const Ctx &c, u32 slot, u32 page, u32 gen, u32 g, 
   {
     const bool have = lane < n;
     const u32 qs = have ? mine / c.WR : 0u, j = have ? mine % c.WR : 0u;
-    consume_group(c, n >= 32 ? 0xffffffffu : ((1u << n) - 1u), qs, j, slot, lane);
+    u32 phase = 0, qid = 0, node = 0;
+    u64 worst = 0;
+    if (have) {
+      const QHdr *h = c.hdr + qs;
+      phase = ld_u32(&h->phase); qid = ld_u32(&h->qid);
+      node = ld_u32(c.items + mine);
+      if (c.stash_cap) worst = ld_u64((const u64 *)&h->worst_lo);
+    }
+    consume_group<PQ>(c, n >= 32 ? 0xffffffffu : ((1u << n) - 1u), qs, j, slot, phase, qid, node, worst, lane);
     // consume_group ends with a warp barrier: every lane's result stores happen before the
     // owner lane's fence + decrement below
     if (have) complete_items(c, qs, 1);
@@ -607,6 +675,7 @@ __device__ void consume_chain(const Ctx &c, u32 slot, u32 page, u32 gen, u32 g, 
 // A page has arrived in `slot` (Section 3.2: the per-slot ready entry): take its waiter
 // list, serve it, then make the page evictable.  v is a slot id, or a continuation
 // (kContFlag | record) of a chain another warp handed off.
+template <bool PQ>
 __device__ void consume_arrival(const Ctx &c, u32 v, u32 lane) {
   if (v & kContFlag) {
     const u32 g = v & ~kContFlag;
@@ -616,7 +685,7 @@ __device__ void consume_arrival(const Ctx &c, u32 v, u32 lane) {
     u64 w = ld_u64(c.ptab + page);
     w = __shfl_sync(0xffffffffu, w, 0);
     if (pw_state(w) != P_ARRIVED) { if (lane == 0) raise(c, 8, 0x75, g, page, (u32)(w >> 32)); return; }
-    consume_chain(c, pw_slot(w), page, pw_low(w), g, lane);
+    consume_chain<PQ>(c, pw_slot(w), page, pw_low(w), g, lane);
     return;
   }
   const u32 slot = v;
@@ -648,7 +717,7 @@ __device__ void consume_arrival(const Ctx &c, u32 v, u32 lane) {
   }
   if (__shfl_sync(0xffffffffu, bad, 0)) return;
   head = __shfl_sync(0xffffffffu, head, 0);
-  consume_chain(c, slot, page, gen, head, lane);
+  consume_chain<PQ>(c, slot, page, gen, head, lane);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -683,10 +752,14 @@ __device__ __forceinline__ void phase_mark(const Ctx &c, u64 &t, u32 idx, u32 la
 // leave the item waiting on the page.  Returns true if the whole batch completed inline
 // (the caller goes on with the next phase), false if the query is parked: whoever
 // consumes its last item pushes it back onto the runnable queue.
-__device__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
+template <bool PQ>
+__device__ __noinline__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
   QHdr *h = c.hdr + qs;
-  const u32 phase = uld(&h->phase);
-  const u32 n = uld(&h->n_items);
+  // qid, phase, (awaiting), n_items sit in the header's first 16 bytes; only this warp writes
+  // them while it runs the query, so every lane may read them for itself
+  const uint4 h0 = ld_v4((const u32 *)h);
+  const u32 qid = h0.x, phase = h0.y, n = h0.w;
+  const u64 worst = c.stash_cap ? ld_u64((const u64 *)&h->worst_lo) : 0ull;
   const bool count_pages = (c.pq_m == 0) == (phase == PH_EVAL);
   if (lane == 0) st_u32(&h->awaiting, n + 1u);      // +1: guard held until everything is issued
   __threadfence();
@@ -701,9 +774,11 @@ __device__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
     const u32 j = base + lane;
     bool pending = j < n;
     u32 node = 0, page = kInvalidId;      // page: the cache unit looked up (see unit_of)
+    u64 w_first = kAbsentWord;
     if (pending) {
       node = ld_u32(items + j);
       page = unit_of(c, node);
+      w_first = ld_u64(c.ptab + page);    // in flight while the page set is probed
       if (count_pages) {                  // distinct index pages, whatever the cache's unit
         const u32 ipage = node / c.npp;
         u32 r = set_insert(pset, c.pset_cap, ipage);
@@ -737,20 +812,20 @@ __device__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
     phase_mark(c, tq, S_I_SETUP, lane);
     for (u32 round = 0; __any_sync(0xffffffffu, pending); ++round) {
       u32 code = LK_NONE, slot = 0, gen = 0;
-      if (pending) code = page_lookup(c, page, qs * c.WR + j, slot, gen, st);
+      if (pending) code = page_lookup(c, page, qs * c.WR + j, round ? ld_u64(c.ptab + page) : w_first, slot, gen, st);
       __syncwarp();
       phase_mark(c, tq, S_I_LOOKUP, lane);
       if (code == LK_WAIT) pending = false;
       const u32 hits = __ballot_sync(0xffffffffu, code == LK_HIT);
-      if (hits) consume_group(c, hits, qs, j, slot, lane);
+      if (hits) consume_group<PQ>(c, hits, qs, j, slot, phase, qid, node, worst, lane);
       if (hits) {
         __threadfence();
         if (code == LK_HIT) {
           // the bytes just read were the page's if its word still names this slot and fill
           const u64 w2 = ld_u64(c.ptab + page);
+          const u64 m2 = ld_u64(c.smeta + slot);          // (for the reference bit; loaded alongside)
           const u32 s2 = pw_state(w2);
           if ((s2 == P_RESIDENT || s2 == P_ARRIVED) && pw_slot(w2) == slot && pw_low(w2) == gen) {
-            const u64 m2 = ld_u64(c.smeta + slot);
             if (!(m2 & 1ull)) atomicCAS((unsigned long long *)(c.smeta + slot), m2, m2 | 1ull);
             st.hit++; n_done++;
             pending = false;
@@ -1190,6 +1265,7 @@ __device__ bool warp_ticket(int *count, u32 *head, u32 &idx, u32 lane);
 // One unit of the work that keeps pages moving, in priority order: execute a copy the proxy
 // has admitted, consume a page the proxy has published (or a handed-off waiter chain), give
 // a waiting page a slot.  Returns 0 if there was nothing to do, 1 for a copy, 2 for an arrival.
+template <bool PQ>
 __device__ __noinline__ u32 service_step(const Ctx &c, u32 lane) {
   u32 v;
   if (warp_ticket(&c.ctl->counts[0], &c.cs->copy_head, v, lane)) {    // the outstanding window waits on these
@@ -1198,11 +1274,11 @@ __device__ __noinline__ u32 service_step(const Ctx &c, u32 lane) {
   }
   if (warp_ticket(&c.ctl->counts[1], &c.cs->comp_head, v, lane)) {    // completion v: its page has arrived
     const u64 e = __shfl_sync(0xffffffffu, ld_u64(c.ring_dev + (v & c.ring_mask)), 0);
-    consume_arrival(c, (u32)(e >> 8) & 0xFFFFFFu, lane);
+    consume_arrival<PQ>(c, (u32)(e >> 8) & 0xFFFFFFu, lane);
     return 2;
   }
   if (warp_pop(c, c.arr, v, lane)) {                                  // handed-off waiter chains
-    consume_arrival(c, v, lane);
+    consume_arrival<PQ>(c, v, lane);
     return 2;
   }
   return 0;
@@ -1221,12 +1297,13 @@ __device__ void idle_step(const Ctx &c, u32 lane) {
 // "issue remote reads and wait for page readiness"): the warp keeps its query and waits in
 // place until the batch it issued is complete.  It still moves pages while it waits -- someone
 // has to -- but it never picks up another query, so at most one query per warp is in flight.
+template <bool PQ>
 __device__ __noinline__ bool wait_in_place(const Ctx &c, u32 qs, u32 lane) {
   const u64 t0 = globaltimer();
   for (u32 it = 0;; ++it) {
     if (uld(&c.hdr[qs].awaiting) == 0u) { __threadfence(); return true; }
     if (warp_stopped(c)) return false;
-    if (service_step(c, lane) == 0) { idle_step(c, lane); __nanosleep(200); }
+    if (service_step<PQ>(c, lane) == 0) { idle_step(c, lane); __nanosleep(200); }
     u32 late = ((it & 255u) == 255u && globaltimer() - t0 > c.timeout_ns) ? 1u : 0u;
     if (__shfl_sync(0xffffffffu, late, 0)) { if (lane == 0) raise(c, 5, 0xB5, qs); return false; }
   }
@@ -1255,9 +1332,9 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut, u32 &lut_qid
         if (lane == 0) st_u64(c.cand + (u64)qs * c.WR, mk_key(lane_adc(c, lut, c.entry), c.entry));
         __syncwarp();
       } else {
-        const bool go = issue_batch(c, qs, lane);
+        const bool go = issue_batch<PQ>(c, qs, lane);
         phase_mark(c, tp, S_P_ISSUE_EVAL, lane);
-        if (!go && !(c.blocking && wait_in_place(c, qs, lane))) return;
+        if (!go && !(c.blocking && wait_in_place<PQ>(c, qs, lane))) return;
       }
     } else if (phase == PH_EVAL) {
       const u32 nf = merge_select_dispatch(c, qs, lane);
@@ -1279,9 +1356,9 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut, u32 &lut_qid
       }
       __syncwarp();
       {
-        const bool go = issue_batch(c, qs, lane);
+        const bool go = issue_batch<PQ>(c, qs, lane);
         phase_mark(c, tp, S_P_ISSUE_EXP, lane);
-        if (!go && !(c.blocking && wait_in_place(c, qs, lane))) return;
+        if (!go && !(c.blocking && wait_in_place<PQ>(c, qs, lane))) return;
       }
     } else {  // PH_EXPAND complete
       const u32 nf = uld(&h->n_items);
@@ -1307,9 +1384,9 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut, u32 &lut_qid
       if (lane == 0) { st_u32(&h->n_items, nn); st_u32(&h->phase, PH_EVAL); }
       __syncwarp();
       if (!PQ && nn > 0) {
-        const bool go = issue_batch(c, qs, lane);
+        const bool go = issue_batch<PQ>(c, qs, lane);
         phase_mark(c, tp, S_P_ISSUE_EVAL, lane);
-        if (!go && !(c.blocking && wait_in_place(c, qs, lane))) return;
+        if (!go && !(c.blocking && wait_in_place<PQ>(c, qs, lane))) return;
       }
     }
   }
@@ -1469,7 +1546,7 @@ __global__ void __launch_bounds__(PQ ? 384 : 768, 1) search_kernel(const Ctx c) 
         continue;
       }
     }
-    if (const u32 what = service_step(c, lane)) {
+    if (const u32 what = service_step<PQ>(c, lane)) {
       idle = 0;
       const u64 t = globaltimer();
       if (what == 1) t_cpy += t - tp; else { t_arr += t - tp; ++n_arr; }
