@@ -76,7 +76,8 @@ enum StatIdx { S_HIT = 0, S_MISSED, S_JOINS, S_EVICT, S_RETRY, S_DONE, S_NEVAL, 
                S_SUMDEG, S_NITER, S_RESUMES, S_POSTED, S_T_ARR, S_T_RUN, S_T_IDLE, S_N_ARR, S_T_CPY, S_STASH,
                // debug profile (Ctx::prof): warp time per query phase step
                S_P_MERGE, S_P_ISSUE_EVAL, S_P_ISSUE_EXP, S_P_COLLECT, S_P_POOL, S_P_LUT, S_P_ADC, S_P_FINISH, S_P_RECYCLE,
-               S_I_SETUP, S_I_LOOKUP, S_I_CONSUME, S_I_TAIL };   // inside issue_batch
+               S_I_SETUP, S_I_LOOKUP, S_I_CONSUME, S_I_TAIL,     // inside issue_batch
+               S_POLLS };                                         // control reads the poller made
 
 // Everything the persistent kernel needs, passed by value.
 struct Ctx {
