@@ -530,21 +530,53 @@ __device__ __noinline__ void consume_group(const Ctx &c, u32 mask, u32 qs, u32 j
   const bool scored = (eval_mask >> lane) & 1u;
   const u64 key = mk_key(dist, node);
   if (scored) st_u64(c.cand + (u64)qs * c.WR + j, key);
-  // adjacency stash for candidates that can still enter the list (see consume_item)
-  for (u32 m = __ballot_sync(0xffffffffu, scored && c.stash_cap && key < worst); m; m &= m - 1) {
-    const u32 src = __ffs(m) - 1;
-    const u32 s_qs = __shfl_sync(0xffffffffu, qs, src), s_node = __shfl_sync(0xffffffffu, node, src);
-    const u32 s_slot = __shfl_sync(0xffffffffu, slot, src);
-    const u32 e = hash32(s_node) & (c.stash_cap - 1);
-    u32 *tag = c.stash_tag + (u64)s_qs * c.stash_cap + e;
-    u32 busy = 0;
-    if (lane == 0) busy = atomicExch(tag, kStashBusy) == kStashBusy ? 1u : 0u;
-    if (!__shfl_sync(0xffffffffu, busy, 0)) {
-      const u32 *adj = (const u32 *)(rec_ptr(c, s_slot, s_node) + c.vec_bytes);
-      u32 *dst = c.stash + ((u64)s_qs * c.stash_cap + e) * (c.R + 1u);
-      for (u32 i = lane; i < c.R + 1u; i += 32) st_u32(dst + i, __ldcg(adj + i));
+  // Adjacency stash for candidates that can still enter the list (see consume_item).  Every
+  // owner lane claims its own entry (all claims in flight together), the warp copies the
+  // claimed lists two at a time with their loads in flight, and the tags are published last.
+  {
+    u32 e = 0;
+    bool own = false;
+    if (scored && c.stash_cap && key < worst) {
+      e = hash32(node) & (c.stash_cap - 1);
+      own = atomicExch(c.stash_tag + (u64)qs * c.stash_cap + e, kStashBusy) != kStashBusy;
+    }
+    const u32 owners = __ballot_sync(0xffffffffu, own);
+    const bool narrow = c.R + 1u <= 96u;
+    for (u32 m = owners; m;) {
+      u32 src[2], a[2][3];
+      int ng = 0;
+#pragma unroll
+      for (int g = 0; g < 2; ++g) { src[g] = 0; if (m && (g == 0 || narrow)) { src[g] = __ffs(m) - 1; m &= m - 1; ng = g + 1; } }
+#pragma unroll
+      for (int g = 0; g < 2; ++g) {
+        if (g < ng) {
+          const u32 s_node = __shfl_sync(0xffffffffu, node, src[g]), s_slot = __shfl_sync(0xffffffffu, slot, src[g]);
+          const u32 *adj = (const u32 *)(rec_ptr(c, s_slot, s_node) + c.vec_bytes);
+          if (narrow) {
+#pragma unroll
+            for (int k = 0; k < 3; ++k) { const u32 i = (u32)k * 32u + lane; a[g][k] = i <= c.R ? __ldcg(adj + i) : 0u; }
+          }
+        }
+      }
+#pragma unroll
+      for (int g = 0; g < 2; ++g) {
+        if (g < ng) {
+          const u32 s_qs = __shfl_sync(0xffffffffu, qs, src[g]), s_e = __shfl_sync(0xffffffffu, e, src[g]);
+          u32 *dst = c.stash + ((u64)s_qs * c.stash_cap + s_e) * (c.R + 1u);
+          if (narrow) {
+#pragma unroll
+            for (int k = 0; k < 3; ++k) { const u32 i = (u32)k * 32u + lane; if (i <= c.R) st_u32(dst + i, a[g][k]); }
+          } else {
+            const u32 s_node = __shfl_sync(0xffffffffu, node, src[g]), s_slot = __shfl_sync(0xffffffffu, slot, src[g]);
+            const u32 *adj = (const u32 *)(rec_ptr(c, s_slot, s_node) + c.vec_bytes);
+            for (u32 i = lane; i < c.R + 1u; i += 32) st_u32(dst + i, __ldcg(adj + i));
+          }
+        }
+      }
+    }
+    if (owners) {
       __syncwarp();
-      if (lane == 0) { __threadfence(); st_u32(tag, s_node); }
+      if (own) { __threadfence(); st_u32(c.stash_tag + (u64)qs * c.stash_cap + e, node); }
     }
   }
   // Expansion items: copy the node's adjacency list into the query's buffer (PQ navigation: also
