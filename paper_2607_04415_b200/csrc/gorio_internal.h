@@ -69,7 +69,7 @@ struct Ctl {
   u32 q_heads[16]; // queue head/tail words: arr(0,1) run(3,4) want(6,7)
   u32 dbg[8];      // detail of the first error
   u32 census[16];  // debug snapshot (see census())
-  u64 stats[32];
+  u64 stats[48];
 };
 
 enum StatIdx { S_HIT = 0, S_MISSED, S_JOINS, S_EVICT, S_RETRY, S_DONE, S_NEVAL, S_NEXPAND,
@@ -77,7 +77,8 @@ enum StatIdx { S_HIT = 0, S_MISSED, S_JOINS, S_EVICT, S_RETRY, S_DONE, S_NEVAL, 
                // debug profile (Ctx::prof): warp time per query phase step
                S_P_MERGE, S_P_ISSUE_EVAL, S_P_ISSUE_EXP, S_P_COLLECT, S_P_POOL, S_P_LUT, S_P_ADC, S_P_FINISH, S_P_RECYCLE,
                S_I_SETUP, S_I_LOOKUP, S_I_CONSUME, S_I_TAIL,     // inside issue_batch
-               S_POLLS };                                         // control reads the poller made
+               S_POLLS,                                           // control reads the poller made
+               S_A_HEAD, S_A_WALK, S_A_GROUP, S_A_COMPLETE, S_A_FINISH };   // inside an arrival
 
 // Everything the persistent kernel needs, passed by value.
 struct Ctx {

@@ -77,6 +77,14 @@ __device__ __forceinline__ u32 uld(const u32 *p) { return __shfl_sync(0xffffffff
 __device__ __forceinline__ void stat_add(const Ctx &c, u32 idx, u32 v) {
   if (v) atomicAdd((unsigned long long *)&c.ctl->stats[idx], (unsigned long long)v);
 }
+// Debug profile: charge the time since `t` to stats[idx] and restart the clock.
+__device__ __forceinline__ void phase_mark(const Ctx &c, u64 &t, u32 idx, u32 lane) {
+  if (!c.prof) return;
+  const u64 now = globaltimer();
+  if (lane == 0) atomicAdd((unsigned long long *)&c.ctl->stats[idx], now - t);
+  t = now;
+}
+
 
 // ------------------------------------------------------------------------------------------
 // bounded MPMC queue of u32 (cells = sequence << 32 | value); one lane calls these
@@ -668,8 +676,10 @@ __device__ void finish_arrival(const Ctx &c, u32 slot, u32 page, u32 gen, u32 la
 
 // Consume the waiter chain starting at record g for the page held in `slot`.
 template <bool PQ>
-__device__ void consume_chain(const Ctx &c, u32 slot, u32 page, u32 gen, u32 g, u32 lane) {
+__device__ void consume_chain(const Ctx &c, u32 slot, u32 page, u32 gen, u32 g, u32 lane, u64 tp = 0) {
   const u32 limit = c.n_qslots * c.WR;
+  if (c.prof && tp == 0) tp = globaltimer();
+  phase_mark(c, tp, S_A_HEAD, lane);
   // chase up to a segment of next pointers first so that the remainder is handed off early
   u32 mine = kNil, n = 0, cur = g;
   while (cur != kNil && n < kChainSegment) {
@@ -682,6 +692,7 @@ __device__ void consume_chain(const Ctx &c, u32 slot, u32 page, u32 gen, u32 g, 
     atomicAdd(c.parts + slot, 1u);
     q_push(c, c.arr, kContFlag | cur);
   }
+  phase_mark(c, tp, S_A_WALK, lane);
   {
     const bool have = lane < n;
     const u32 qs = have ? mine / c.WR : 0u, j = have ? mine % c.WR : 0u;
@@ -694,14 +705,17 @@ __device__ void consume_chain(const Ctx &c, u32 slot, u32 page, u32 gen, u32 g, 
       if (c.stash_cap) worst = ld_u64((const u64 *)&h->worst_lo);
     }
     consume_group<PQ>(c, n >= 32 ? 0xffffffffu : ((1u << n) - 1u), qs, j, slot, phase, qid, node, worst, lane);
+    phase_mark(c, tp, S_A_GROUP, lane);
     // consume_group ends with a warp barrier: every lane's result stores happen before the
     // owner lane's fence + decrement below
     if (have) complete_items(c, qs, 1);
     __syncwarp();
+    phase_mark(c, tp, S_A_COMPLETE, lane);
   }
   u32 last = 0;
   if (lane == 0) last = atomicSub(c.parts + slot, 1u) == 1u ? 1u : 0u;
   if (__shfl_sync(0xffffffffu, last, 0)) finish_arrival(c, slot, page, gen, lane);
+  phase_mark(c, tp, S_A_FINISH, lane);
 }
 
 // A page has arrived in `slot` (Section 3.2: the per-slot ready entry): take its waiter
@@ -722,6 +736,7 @@ __device__ void consume_arrival(const Ctx &c, u32 v, u32 lane) {
   }
   const u32 slot = v;
   if (slot >= c.n_slots) { if (lane == 0) raise(c, 8, 0x71, slot); return; }
+  const u64 tp = c.prof ? globaltimer() : 0;
   u64 m = ld_u64(c.smeta + slot);
   m = __shfl_sync(0xffffffffu, m, 0);
   const u32 page = sm_page(m), gen = sm_gen(m);
@@ -749,7 +764,7 @@ __device__ void consume_arrival(const Ctx &c, u32 v, u32 lane) {
   }
   if (__shfl_sync(0xffffffffu, bad, 0)) return;
   head = __shfl_sync(0xffffffffu, head, 0);
-  consume_chain<PQ>(c, slot, page, gen, head, lane);
+  consume_chain<PQ>(c, slot, page, gen, head, lane, tp);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -766,14 +781,6 @@ __device__ u32 set_insert(u32 *tab, u32 cap, u32 v) {
     h = (h + 1) & (cap - 1);
   }
   return 2;
-}
-
-// Debug profile: charge the time since `t` to stats[idx] and restart the clock.
-__device__ __forceinline__ void phase_mark(const Ctx &c, u64 &t, u32 idx, u32 lane) {
-  if (!c.prof) return;
-  const u64 now = globaltimer();
-  if (lane == 0) atomicAdd((unsigned long long *)&c.ctl->stats[idx], now - t);
-  t = now;
 }
 
 // ------------------------------------------------------------------------------------------
