@@ -160,6 +160,40 @@ def test_single_query_and_unreachable_results_are_padded(gorio):
         ix.close()
 
 
+def test_empty_batch_is_rejected_and_one_node_index_works(gorio):
+    """Degenerate inputs: no queries (an argument error, nothing launched), an index of a single
+    node without edges, and a two-node index whose lists hold self loops and duplicates."""
+    pages1 = write_page_store(np.array([[7, 7, 7, 7]], dtype=np.uint8), np.zeros(1, np.uint32),
+                              np.full((1, 3), 0xFFFFFFFF, np.uint32), 1)
+    ix = gorio.Index(pages1, 1, 4, "u8", 3, 1, 0)
+    try:
+        ix.cache_config(16)
+        with pytest.raises(gorio.GorioError) as e:
+            ix.search(torch.zeros((0, 4), dtype=torch.uint8).cuda(), 1, 1, 1)
+        assert e.value.status == 1
+        q = torch.tensor([[7, 7, 7, 9], [0, 0, 0, 0]], dtype=torch.uint8).cuda()
+        out = ix.search(q, 2, 4, 2)
+        assert _u32(out["ids"]).tolist() == [[0, 0xFFFFFFFF], [0, 0xFFFFFFFF]]
+        assert _u32(out["dists"]).tolist() == [[4, 0xFFFFFFFF], [196, 0xFFFFFFFF]]
+        assert _u32(out["counters"]).tolist() == [[1, 1, 1, 1, 0]] * 2
+    finally:
+        ix.close()
+    data = np.array([[0, 0, 0, 0], [3, 0, 0, 0]], dtype=np.uint8)
+    deg = np.array([3, 3], dtype=np.uint32)
+    nbrs = np.array([[0, 1, 1], [1, 1, 0]], dtype=np.uint32)           # self loops and duplicates
+    pages2 = write_page_store(data, deg, nbrs, 2)
+    ref = OracleIndex(pages2, 2, 4, "u8", 3, 2, 0).search(np.array([[2, 0, 0, 0]], dtype=np.uint8), 2, 2, 1)
+    ix = gorio.Index(pages2, 2, 4, "u8", 3, 2, 0)
+    try:
+        ix.cache_config(16)
+        out = ix.search(torch.tensor([[2, 0, 0, 0]], dtype=torch.uint8).cuda(), 2, 2, 1)
+        assert (_u32(out["ids"]) == ref["ids"]).all() and (_u32(out["dists"]) == ref["dists"]).all()
+        assert (_u32(out["counters"]) == ref["counters"]).all()
+        assert _u32(out["ids"]).tolist() == [[1, 0]] and _u32(out["dists"]).tolist() == [[1, 4]]
+    finally:
+        ix.close()
+
+
 def test_ring_worked_example_on_gpu(gorio):
     from helpers import ring_index
     data, deg, nbrs, pages = ring_index([10 * i for i in range(8)], d=4, npp=2)
