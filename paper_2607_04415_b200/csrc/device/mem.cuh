@@ -42,6 +42,7 @@ __device__ __forceinline__ u64 globaltimer() {
   u64 t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t;
 }
 __device__ __forceinline__ u32 lane_id() { return threadIdx.x & 31u; }
+__device__ __forceinline__ u32 hash32(u32 v) { v *= 0x9E3779B1u; v ^= v >> 15; return v * 0x85EBCA77u; }
 
 // ------------------------------------------------------------------------------------------
 // errors and statistics

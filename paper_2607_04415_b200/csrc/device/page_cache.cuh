@@ -135,36 +135,46 @@ __device__ void serve_want(const Ctx &c, u32 hint, LaneStats &st) {
 enum LookupCode : u32 { LK_NONE = 0, LK_HIT = 1, LK_WAIT = 2 };
 // `first` is the page word as the caller last saw it (every decision below is re-checked by a
 // compare-and-swap or by the caller's validation, so a stale word only costs a retry).
+//
+// Joining a waiter list is a compare-and-swap on the page word, and a batch starts with every
+// query joining the entry node's page at once: thousands of lanes retry against one word, and
+// every success makes all other attempts in flight fail.  The loop is lock-free (some lane
+// always gets through), so the retry bound is generous; a failed attempt continues from the
+// word the compare-and-swap returned instead of re-reading it, and backs off for a short,
+// per-lane pseudo-random time once it has failed a few times.  (A bound of 4,096 attempts
+// without back-off was exceeded once in some two hundred full-size searches.)
+constexpr u32 kLookupTries = 1u << 20;
 __device__ u32 page_lookup(const Ctx &c, u32 page, u32 g, u64 first, u32 &slot, u32 &gen, LaneStats &st) {
   u64 *pw = c.ptab + page;
-  for (u32 tries = 0; tries < 4096; ++tries) {
-    const u64 w = tries ? ld_u64(pw) : first;
+  u64 w = first;
+  for (u32 tries = 0; tries < kLookupTries; ++tries) {
     const u32 s = pw_state(w);
     if (s == P_RESIDENT || s == P_ARRIVED) { slot = pw_slot(w); gen = pw_low(w); return LK_HIT; }
     st_u32(c.wrec + g, s == P_ABSENT ? kNil : pw_low(w));
     __threadfence();
-    if (s == P_ABSENT) {
-      const u64 wanted = mk_pw(P_WANTED, 0, g);
-      if (atomicCAS((unsigned long long *)pw, w, wanted) != w) continue;
-      st.missed++;
-      // First requester: find the page a slot -- but never ahead of pages that already wait for
-      // one.  Requests leave in the order in which their pages were first wanted, so each has
-      // gathered as many waiters as it can by the time it is posted; letting new pages jump the
-      // queue whenever the backlog had room cost 16 % more fetches on config 3.
-      const bool room = may_post(c);
-      const bool queued = (int)ld_u32((const u32 *)c.want.count) > 0;
-      u32 prev_gen = 0;
-      const u32 sl = (room && !queued) ? alloc_slot(c, kNil, st, prev_gen) : kNil;
-      if (sl != kNil) {
-        assign_and_post(c, page, sl, prev_gen, wanted, st);
-      } else {
-        q_push(c, c.want, page);
-        if (room) serve_want(c, kNil, st);      // the oldest waiting page takes the opening
-      }
-      return LK_WAIT;
+    const u64 mine = s == P_ABSENT ? mk_pw(P_WANTED, 0, g) : ((w & 0xFFFFFFFF00000000ull) | g);
+    const u64 old = atomicCAS((unsigned long long *)pw, w, mine);
+    if (old != w) {                                   // lost the race: `old` is the word as it is now
+      w = old;
+      if (tries >= 4) __nanosleep(32u * (tries < 32u ? tries : 32u) + (hash32(g + tries) & 1023u));
+      continue;
     }
-    if (atomicCAS((unsigned long long *)pw, w, (w & 0xFFFFFFFF00000000ull) | g) != w) continue;
-    st.missed++; st.joins++;
+    st.missed++;
+    if (s != P_ABSENT) { st.joins++; return LK_WAIT; }
+    // First requester: find the page a slot -- but never ahead of pages that already wait for
+    // one.  Requests leave in the order in which their pages were first wanted, so each has
+    // gathered as many waiters as it can by the time it is posted; letting new pages jump the
+    // queue whenever the backlog had room cost 16 % more fetches on config 3.
+    const bool room = may_post(c);
+    const bool queued = (int)ld_u32((const u32 *)c.want.count) > 0;
+    u32 prev_gen = 0;
+    const u32 sl = (room && !queued) ? alloc_slot(c, kNil, st, prev_gen) : kNil;
+    if (sl != kNil) {
+      assign_and_post(c, page, sl, prev_gen, mine, st);
+    } else {
+      q_push(c, c.want, page);
+      if (room) serve_want(c, kNil, st);      // the oldest waiting page takes the opening
+    }
     return LK_WAIT;
   }
   raise(c, 8, 0x42, page, g);

@@ -39,7 +39,6 @@ __device__ __forceinline__ u32 key_id(u64 k) { return (u32)(k & 0xFFFFFFFFull) >
 __device__ __forceinline__ u32 key_dist(u64 k) { return (u32)(k >> 32); }
 
 constexpr u32 kStashBusy = 0xFFFFFFFEu;
-__device__ __forceinline__ u32 hash32(u32 v) { v *= 0x9E3779B1u; v ^= v >> 15; return v * 0x85EBCA77u; }
 
 // Consume item j of query slot qs from the page in `slot` (warp cooperative).
 //   PH_EVAL   : score the node, write its key into the candidate buffer.

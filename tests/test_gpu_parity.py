@@ -433,6 +433,26 @@ def test_queries_not_16_byte_aligned_take_the_narrow_path(gorio, cfg1):
         ix.close()
 
 
+def test_sixteen_thousand_queries_join_the_entry_page_at_once_repeatedly(gorio, cfg1):
+    """Every query's first item is the entry node, so a batch opens with all of its queries
+    joining one page's waiter list through compare-and-swap on one word.  Ten cold searches of
+    16,384 queries each must all come out exact."""
+    w, ref = cfg1
+    reps = -(-16384 // w.nq)
+    q = np.tile(w.queries, (reps, 1))[:16384]
+    rows = np.arange(16384) % w.nq
+    ix = gorio.Index.from_workload(w)
+    try:
+        qd = torch.as_tensor(q).cuda()
+        for it in range(10):
+            ix.cache_config(500, remote_latency_ns=(0, 20000)[it % 2], max_outstanding=256, timeout_ms=60000)
+            out = ix.search(qd, w.K, w.L, w.W)
+            assert (_u32(out["ids"]) == ref["ids"][rows]).all()
+            assert (_u32(out["counters"]) == ref["counters"][rows]).all()
+    finally:
+        ix.close()
+
+
 def test_second_search_reuses_the_warm_cache(gorio, cfg1):
     w, ref = cfg1
     ix = gorio.Index.from_workload(w)
