@@ -27,14 +27,25 @@ def build(force: bool = False, verbose: bool = False) -> str:
     """Compile csrc/*.cu into libgorio.so next to this file (nvcc cross-compiles without a GPU)."""
     if not force and not _stale():
         return LIB_PATH
-    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    objs = []
-    for src in SOURCES:
-        obj = os.path.join(CSRC, src.replace(".cu", ".o"))
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", os.path.join(CSRC, src), "-o", obj]
-        subprocess.check_call(cmd)
-        objs.append(obj)
-    subprocess.check_call([nvcc, "-shared", "-o", LIB_PATH] + objs + ["-lcudart"])
+    # one builder at a time: ranks of a multi-process launch may all find the library stale
+    import fcntl
+    with open(os.path.join(_HERE, ".build.lock"), "w") as lock:
+        fcntl.flock(lock, fcntl.LOCK_EX)
+        try:
+            if not force and not _stale():      # another process built it while this one waited
+                return LIB_PATH
+            nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+            objs = []
+            for src in SOURCES:
+                obj = os.path.join(CSRC, src.replace(".cu", ".o"))
+                cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", os.path.join(CSRC, src), "-o", obj]
+                subprocess.check_call(cmd)
+                objs.append(obj)
+            tmp = LIB_PATH + ".tmp"
+            subprocess.check_call([nvcc, "-shared", "-o", tmp] + objs + ["-lcudart"])
+            os.replace(tmp, LIB_PATH)           # readers never see a half-written library
+        finally:
+            fcntl.flock(lock, fcntl.LOCK_UN)
     return LIB_PATH
 
 
