@@ -16,11 +16,25 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
               "-Xcompiler", "-fPIC", "-Xcompiler", "-pthread"]
 
 
+STAMP_PATH = LIB_PATH + ".stamp"      # hash of the sources and flags the library was built from
+
+
+def _source_hash() -> str:
+    import hashlib
+    h = hashlib.sha256(" ".join(NVCC_FLAGS).encode())
+    for f in SOURCES + HEADERS:
+        with open(os.path.join(CSRC, f), "rb") as fh:
+            h.update(f.encode() + b"\0" + fh.read())
+    return h.hexdigest()
+
+
 def _stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+    """True unless the library was built from exactly these sources (file times do not survive a
+    copy of the tree to another machine, contents do)."""
+    if not (os.path.exists(LIB_PATH) and os.path.exists(STAMP_PATH)):
         return True
-    t = os.path.getmtime(LIB_PATH)
-    return any(os.path.getmtime(os.path.join(CSRC, f)) > t for f in SOURCES + HEADERS)
+    with open(STAMP_PATH) as fh:
+        return fh.read().strip() != _source_hash()
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -44,6 +58,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
             tmp = LIB_PATH + ".tmp"
             subprocess.check_call([nvcc, "-shared", "-o", tmp] + objs + ["-lcudart"])
             os.replace(tmp, LIB_PATH)           # readers never see a half-written library
+            with open(STAMP_PATH, "w") as fh:
+                fh.write(_source_hash())
         finally:
             fcntl.flock(lock, fcntl.LOCK_UN)
     return LIB_PATH
