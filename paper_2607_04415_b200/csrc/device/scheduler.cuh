@@ -215,6 +215,7 @@ __device__ void copy_page(const Ctx &c, u32 idx, u32 lane) {
   }
   uint4 *dst = (uint4 *)(c.slot_data + (u64)slot * c.slot_bytes);
   uint4 v[8];
+  const u64 t_issue = c.prof ? globaltimer() : 0;
 #pragma unroll
   for (int i = 0; i < 8; ++i) v[i] = (u32)i * 32u + lane < chunks ? __ldcs(src + i * 32 + lane) : make_uint4(0, 0, 0, 0);
   // The acknowledgement carries a checksum of the page above the lap tag (the host looks at the
@@ -225,6 +226,7 @@ __device__ void copy_page(const Ctx &c, u32 idx, u32 lane) {
   for (int i = 0; i < 8; ++i) sum ^= v[i].x ^ v[i].y ^ v[i].z ^ v[i].w;
   sum = __reduce_xor_sync(0xffffffffu, sum);
   if (lane == 0) st_sys_u32(c.fdone + (idx & c.ring_mask), ((u32)cmd & 0xFFu) | (sum << 8));
+  if (c.prof && lane == 0) atomicAdd((unsigned long long *)&c.ctl->stats[S_C_DATA], globaltimer() - t_issue);
 #pragma unroll
   for (int i = 0; i < 8; ++i) if ((u32)i * 32u + lane < chunks) __stcg(dst + i * 32 + lane, v[i]);
   __syncwarp();          // orders every lane's stores before lane 0's release below

@@ -609,7 +609,8 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
                            "(issue: setup", "lookup", "consume", "tail)"};
     std::fprintf(stderr, "[gorio profile] warp ms per query step (cumulative since stats_reset):");
     for (int i = 0; i < 13; ++i) std::fprintf(stderr, " %s %.1f", names[i], h.stats[S_P_MERGE + i] / 1e6);
-    std::fprintf(stderr, " | control reads %llu", (unsigned long long)h.stats[S_POLLS]);
+    std::fprintf(stderr, " | control reads %llu | copies: loads issued -> bytes arrived %.1f",
+                 (unsigned long long)h.stats[S_POLLS], h.stats[S_C_DATA] / 1e6);
     std::fprintf(stderr, " | arrival: head %.1f walk %.1f group %.1f complete %.1f finish %.1f", h.stats[S_A_HEAD] / 1e6,
                  h.stats[S_A_WALK] / 1e6, h.stats[S_A_GROUP] / 1e6, h.stats[S_A_COMPLETE] / 1e6, h.stats[S_A_FINISH] / 1e6);
     std::fprintf(stderr, " | arrivals %.1f copies %.1f queries %.1f idle %.1f\n", h.stats[S_T_ARR] / 1e6, h.stats[S_T_CPY] / 1e6,

@@ -78,7 +78,8 @@ enum StatIdx { S_HIT = 0, S_MISSED, S_JOINS, S_EVICT, S_RETRY, S_DONE, S_NEVAL, 
                S_P_MERGE, S_P_ISSUE_EVAL, S_P_ISSUE_EXP, S_P_COLLECT, S_P_POOL, S_P_LUT, S_P_ADC, S_P_FINISH, S_P_RECYCLE,
                S_I_SETUP, S_I_LOOKUP, S_I_CONSUME, S_I_TAIL,     // inside issue_batch
                S_POLLS,                                           // control reads the poller made
-               S_A_HEAD, S_A_WALK, S_A_GROUP, S_A_COMPLETE, S_A_FINISH };   // inside an arrival
+               S_A_HEAD, S_A_WALK, S_A_GROUP, S_A_COMPLETE, S_A_FINISH,     // inside an arrival
+               S_C_DATA };                                        // copy: loads issued -> bytes in registers
 
 // Everything the persistent kernel needs, passed by value.
 struct Ctx {
