@@ -3,6 +3,9 @@
 // remote tier (paper Section 3.3: the proxy "batches submissions and completions, controls
 // outstanding remote I/O, and publishes ready state", and never looks at search state).
 #include <atomic>
+#if defined(__x86_64__) || defined(__i386__)
+#include <immintrin.h>
+#endif
 #include <chrono>
 #include <condition_variable>
 #include <cstdio>
@@ -102,10 +105,20 @@ int cuda_fail(gorio_index *ix, cudaError_t e, const char *what) {
     if (e__ != cudaSuccess) return cuda_fail(ix, e__, #call);            \
   } while (0)
 
+// Flush the CPU's write-combining buffers (the control block the GPU polls is write-combined
+// memory: written by the proxy, never read by it, and read over PCIe without a cache snoop).
+inline void flush_wc() {
+#if defined(__x86_64__) || defined(__i386__)
+  _mm_sfence();
+#else
+  std::atomic_thread_fence(std::memory_order_seq_cst);
+#endif
+}
+
 template <typename T>
-cudaError_t host_mapped(T **h, T **d, size_t count) {
+cudaError_t host_mapped(T **h, T **d, size_t count, unsigned extra_flags = 0) {
   void *p = nullptr;
-  cudaError_t e = cudaHostAlloc(&p, count * sizeof(T), cudaHostAllocMapped | cudaHostAllocPortable);
+  cudaError_t e = cudaHostAlloc(&p, count * sizeof(T), cudaHostAllocMapped | cudaHostAllocPortable | extra_flags);
   if (e != cudaSuccess) return e;
   std::memset(p, 0, count * sizeof(T));
   *h = (T *)p;
@@ -186,6 +199,7 @@ void proxy_service(gorio_index *ix) {
     }
     if (admitted) {
       hctl[2] = tail;                             // requests [0, tail) may be copied now
+      flush_wc();
       ++batches;
       if (outstanding > max_seen) max_seen = outstanding;
     }
@@ -208,6 +222,7 @@ void proxy_service(gorio_index *ix) {
       }
       if (published) {
         hctl[0] = ct;                             // completions [0, ct) are published, in ring order
+        flush_wc();
         outstanding -= published;
         fetched += published;
       }
@@ -429,7 +444,7 @@ int gorio_index_open(const gorio_index_desc *d, int cuda_device, gorio_index **o
   if (cudaHostGetDevicePointer(&dp, (void *)d->host_pages, 0) != cudaSuccess) return bail(GORIO_ERR_CUDA);
   ix->pages_dev = (const u8 *)dp;
   if (preload_kernels() != cudaSuccess) return bail(GORIO_ERR_CUDA);
-  if (host_mapped(&ix->hctl_h, &ix->hctl_d, 64) != cudaSuccess) return bail(GORIO_ERR_CUDA);
+  if (host_mapped(&ix->hctl_h, &ix->hctl_d, 64, cudaHostAllocWriteCombined) != cudaSuccess) return bail(GORIO_ERR_CUDA);
   if (cudaMalloc(&ix->ctl, sizeof(Ctl)) != cudaSuccess) return bail(GORIO_ERR_NOMEM);
   cudaMemset(ix->ctl, 0, sizeof(Ctl));
   if (cudaStreamCreateWithFlags(&ix->own_stream, cudaStreamNonBlocking) != cudaSuccess) return bail(GORIO_ERR_CUDA);
@@ -572,6 +587,7 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   std::memset(ix->ring_h, 0, (size_t)ix->ring_cap * 8);
   std::memset(ix->fdone_h, 0, (size_t)ix->ring_cap * 4);
   std::memset(ix->hctl_h, 0, 64 * 4);
+  flush_wc();
   std::atomic_thread_fence(std::memory_order_seq_cst);
 
   CK(cudaMemsetAsync(c.seen, 0xFF, (size_t)c.n_qslots * c.seen_cap * 4, stream));
@@ -589,8 +605,8 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   bool host_abort = false;
   cudaError_t qe;
   while ((qe = cudaEventQuery(ix->done_ev)) == cudaErrorNotReady) {
-    if (ix->px_error.load() && !host_abort) { ((volatile u32 *)ix->hctl_h)[1] = 1; host_abort = true; }
-    if (!host_abort && Clock::now() > deadline) { ((volatile u32 *)ix->hctl_h)[1] = 1; host_abort = true; }
+    if (ix->px_error.load() && !host_abort) { ((volatile u32 *)ix->hctl_h)[1] = 1; flush_wc(); host_abort = true; }
+    if (!host_abort && Clock::now() > deadline) { ((volatile u32 *)ix->hctl_h)[1] = 1; flush_wc(); host_abort = true; }
     std::this_thread::sleep_for(std::chrono::microseconds(20));
   }
   proxy_stop(ix);
