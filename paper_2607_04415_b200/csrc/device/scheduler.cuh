@@ -283,17 +283,18 @@ __device__ void poller(const Ctx &c, u32 lane) {
   const u64 t0 = globaltimer();
   bool census_done = c.census_ns == 0;
   for (;;) {
-    if (warp_stopped(c)) break;
     if (!census_done && globaltimer() - t0 > c.census_ns) { census(c, lane); census_done = true; }
-    u32 pub = 0, abort_req = 0, adm = 0;
+    u32 pub = 0, abort_req = 0, adm = 0, stop = 0;
     if (lane == 0) {
-      const uint4 h = ld_sys_v4(c.host_ctl);
+      const uint4 h = ld_sys_v4(c.host_ctl);       // ~6 us under load; the stop flag's load rides along
+      stop = ld_u32(&c.ctl->stop);
       pub = h.x; abort_req = h.y; adm = h.z;
       if (adm != seen_adm) atomicAdd(&c.ctl->counts[0], (int)(adm - seen_adm));
       if (pub != seen_pub) atomicAdd(&c.ctl->counts[1], (int)(pub - seen_pub));
       if (adm == seen_adm && pub == seen_pub) __nanosleep(100);
       seen_adm = adm; seen_pub = pub;
     }
+    if (__shfl_sync(0xffffffffu, stop, 0)) break;
     abort_req = __shfl_sync(0xffffffffu, abort_req, 0);
     if (abort_req) { if (lane == 0) raise(c, 5, 0xB1); break; }
     u32 late = ((++it & 63u) == 0 && globaltimer() - t0 > c.timeout_ns) ? 1u : 0u;
