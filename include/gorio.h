@@ -13,7 +13,10 @@
  *   - "device" pointers are CUDA device memory of the index's device; "host" pointers
  *     are ordinary host memory.  No torch or C++ types cross this boundary.
  *   - The library needs its CUDA kernels: there is no CPU fallback of any kind.
- *   - A gorio_index is not thread safe; use one caller thread per index.
+ *   - Calls on one gorio_index are serialised by the library (a search blocks other callers of
+ *     that index until it returns); different indexes are independent.  gorio_index_close must
+ *     not race with any other call on the same handle.  gorio_last_error returns a pointer
+ *     into the index that the next failing call overwrites.
  */
 #ifndef GORIO_H
 #define GORIO_H

@@ -71,6 +71,8 @@ struct gorio_index {
   void *st_q = nullptr; size_t st_q_bytes = 0;
   void *st_out = nullptr; size_t st_out_bytes = 0;
 
+  std::recursive_mutex api_mu;   // calls on one index are serialised (search_host calls search)
+
   // proxy
   std::thread proxy;
   std::mutex mu;
@@ -481,6 +483,7 @@ int gorio_index_close(gorio_index *ix) {
 
 int gorio_cache_config(gorio_index *ix, const gorio_cache_cfg *cfg) {
   if (!ix || !cfg) return GORIO_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> api_lock(ix->api_mu);
   if (cfg->capacity_pages < 16 || cfg->max_outstanding < 1)
     return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: capacity >= 16, max_outstanding >= 1");
   if (cfg->granularity > GORIO_GRAN_RECORD) return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: unknown granularity");
@@ -500,6 +503,7 @@ int gorio_cache_config(gorio_index *ix, const gorio_cache_cfg *cfg) {
 
 int gorio_set_tuning(gorio_index *ix, const gorio_tuning *t) {
   if (!ix || !t) return GORIO_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> api_lock(ix->api_mu);
   if (t->visited_capacity && ((t->visited_capacity & (t->visited_capacity - 1)) || t->visited_capacity < 64))
     return fail(ix, GORIO_ERR_INVALID_ARG, "visited_capacity must be a power of two >= 64");
   if (t->warps_per_block > 24) return fail(ix, GORIO_ERR_INVALID_ARG, "warps_per_block <= 24");
@@ -513,6 +517,7 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
                  uint32_t *out_ids_dev, void *out_dists_dev, uint32_t *out_pages_distinct_dev,
                  uint32_t *out_counters_dev, void *cuda_stream) {
   if (!ix) return GORIO_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> api_lock(ix->api_mu);
   if (!queries_dev || !out_ids_dev || !out_dists_dev || nq < 1 || K < 1 || K > L || L > 256 || W < 1 ||
       W > 16 || (u64)W * ix->desc.max_degree > 1024)
     return fail(ix, GORIO_ERR_INVALID_ARG, "search: need 1 <= K <= L <= 256, 1 <= W <= 16, W*max_degree <= 1024");
@@ -653,6 +658,7 @@ int gorio_search_host(gorio_index *ix, const void *queries_host, uint32_t nq, ui
                       uint32_t *out_ids_host, void *out_dists_host, uint32_t *out_pages_distinct_host,
                       uint32_t *out_counters_host) {
   if (!ix || !queries_host || !out_ids_host || !out_dists_host || nq < 1 || K < 1) return GORIO_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> api_lock(ix->api_mu);
   CK(cudaSetDevice(ix->dev));
   const size_t qb = (size_t)nq * ix->vec_bytes;
   const size_t ob = (size_t)nq * K * 8 + (size_t)nq * 4 + (size_t)nq * 20;
@@ -676,6 +682,7 @@ int gorio_search_host(gorio_index *ix, const void *queries_host, uint32_t nq, ui
 
 int gorio_stats(gorio_index *ix, gorio_stats_t *out) {
   if (!ix || !out) return GORIO_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> api_lock(ix->api_mu);
   CK(cudaSetDevice(ix->dev));
   Ctl h{};
   CK(cudaMemcpy(&h, ix->ctl, sizeof(Ctl), cudaMemcpyDeviceToHost));
@@ -697,6 +704,7 @@ int gorio_stats(gorio_index *ix, gorio_stats_t *out) {
 
 int gorio_stats_reset(gorio_index *ix) {
   if (!ix) return GORIO_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> api_lock(ix->api_mu);
   CK(cudaSetDevice(ix->dev));
   CK(cudaMemset((u8 *)ix->ctl + offsetof(Ctl, stats), 0, sizeof(((Ctl *)0)->stats)));
   ix->host_fetched_bytes = 0;

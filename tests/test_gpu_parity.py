@@ -453,6 +453,38 @@ def test_sixteen_thousand_queries_join_the_entry_page_at_once_repeatedly(gorio, 
         ix.close()
 
 
+def test_two_threads_on_one_index_are_serialised(gorio, cfg1):
+    """Calls on one index are serialised by the library: two caller threads searching at the
+    same time both get the oracle's answers."""
+    import threading
+    w, ref = cfg1
+    ix = gorio.Index.from_workload(w)
+    results, errors = {}, []
+    try:
+        ix.cache_config(1000, remote_latency_ns=5000)
+        q = torch.as_tensor(w.queries).cuda()
+
+        def work(tag):
+            try:
+                for _ in range(3):
+                    s = torch.cuda.Stream()
+                    out = ix.search(q, w.K, w.L, w.W, stream=s)
+                    s.synchronize()
+                    results.setdefault(tag, []).append(_u32(out["ids"]).copy())
+            except Exception as e:                       # noqa: BLE001
+                errors.append(e)
+
+        ts = [threading.Thread(target=work, args=(i,)) for i in range(2)]
+        for t in ts:
+            t.start()
+        for t in ts:
+            t.join()
+    finally:
+        ix.close()
+    assert not errors, errors
+    assert all((ids == ref["ids"]).all() for tag in results for ids in results[tag]) and len(results) == 2
+
+
 def test_second_search_reuses_the_warm_cache(gorio, cfg1):
     w, ref = cfg1
     ix = gorio.Index.from_workload(w)
