@@ -58,7 +58,13 @@ __device__ __noinline__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
       w_first = ld_u64(c.ptab + page);    // in flight while the page set is probed
       if (count_pages) {                  // distinct index pages, whatever the cache's unit
         const u32 ipage = node / c.npp;
-        u32 r = set_insert(pset, c.pset_cap, ipage);
+        u32 r;
+        if (c.pset_bitmap) {             // one bit per index page: no probing, and the table stays in L2
+          const u32 bit = 1u << (ipage & 31u);
+          r = (atomicOr(pset + (ipage >> 5), bit) & bit) ? 0u : 1u;
+        } else {
+          r = set_insert(pset, c.pset_cap, ipage);
+        }
         if (r == 1) new_pages++;
         else if (r == 2) raise(c, 6, 0x81, qs, ipage);
       }

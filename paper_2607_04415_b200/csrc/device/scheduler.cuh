@@ -48,7 +48,8 @@ __device__ bool recycle_slot(const Ctx &c, u32 qs, u32 lane) {
   uint4 *s4 = (uint4 *)(c.seen + (u64)qs * c.seen_cap);
   for (u32 i = lane; i < c.seen_cap / 4; i += 32) __stcg(s4 + i, ff);
   uint4 *p4 = (uint4 *)(c.pset + (u64)qs * c.pset_cap);
-  for (u32 i = lane; i < c.pset_cap / 4; i += 32) __stcg(p4 + i, ff);
+  const uint4 pclear = c.pset_bitmap ? make_uint4(0, 0, 0, 0) : ff;
+  for (u32 i = lane; i < c.pset_cap / 4; i += 32) __stcg(p4 + i, pclear);
   uint4 *t4 = (uint4 *)(c.stash_tag + (u64)qs * c.stash_cap);
   for (u32 i = lane; i < c.stash_cap / 4; i += 32) __stcg(t4 + i, ff);
   if (lane == 0) reset_hdr(c.hdr + qs, nxt);

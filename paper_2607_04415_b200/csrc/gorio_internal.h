@@ -120,11 +120,12 @@ struct Ctx {
   u32 *adj;      // [n_qslots][W][R]
   u32 *adjdeg;   // [n_qslots][W]
   u32 *seen;     // [n_qslots][seen_cap]
-  u32 *pset;     // [n_qslots][pset_cap]
+  u32 *pset;     // [n_qslots][pset_cap]   distinct index pages touched: hash set, or bitmap (pset_bitmap)
   u64 *pool;     // [n_qslots][K + W]   PQ rerank pool (sorted, <= K kept)
   u32 *stash;     // [n_qslots][stash_cap][R + 1] adjacency lists kept from scoring time (exact mode)
   u32 *stash_tag; // [n_qslots][stash_cap] node id of each stash entry (all ones = empty)
   u32 seen_cap, pset_cap, stash_cap;
+  u32 pset_bitmap;   // 1: the page set is a bitmap over index pages (pset_cap words) instead of a hash set
   const void *queries;
   u32 *out_ids;
   void *out_dists;
