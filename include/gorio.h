@@ -119,7 +119,9 @@ enum { GORIO_GRAN_PAGE = 0, GORIO_GRAN_RECORD = 1 };
  * Scheduler tuning; all zero = defaults.
  *   max_inflight     query slots resident at once (pending/running queries); default 16384.
  *   visited_capacity per-query exact visited-set entries (power of two), default 32768;
- *                    a query that scores more nodes fails with GORIO_ERR_CAPACITY.
+ *                    a query that scores more nodes fails with GORIO_ERR_CAPACITY.  When a
+ *                    bitmap over all nodes needs no more memory than that (n_nodes / 32 words
+ *                    <= visited_capacity), the bitmap is used instead and can never fill up.
  *   warps_per_block / blocks_per_sm  launch geometry of the persistent kernel (<= 24 warps; with
  *                    PQ navigation at most 12, fewer if the per-warp tables do not fit).
  *   stash_entries    per-query adjacency stash (exact navigation): entries of a direct-mapped

@@ -20,6 +20,11 @@ __device__ u32 set_insert(u32 *tab, u32 cap, u32 v) {
   }
   return 2;
 }
+// the same over a bitmap (one bit per possible value): never full
+__device__ __forceinline__ u32 bit_insert(u32 *bits, u32 v) {
+  const u32 bit = 1u << (v & 31u);
+  return (atomicOr(bits + (v >> 5), bit) & bit) ? 0u : 1u;
+}
 
 // ------------------------------------------------------------------------------------------
 // issue a batch of page items for query slot qs
@@ -60,8 +65,7 @@ __device__ __noinline__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
         const u32 ipage = node / c.npp;
         u32 r;
         if (c.pset_bitmap) {             // one bit per index page: no probing, and the table stays in L2
-          const u32 bit = 1u << (ipage & 31u);
-          r = (atomicOr(pset + (ipage >> 5), bit) & bit) ? 0u : 1u;
+          r = bit_insert(pset, ipage);
         } else {
           r = set_insert(pset, c.pset_cap, ipage);
         }

@@ -217,7 +217,7 @@ __device__ u32 collect_neighbors(const Ctx &c, u32 qs, u32 lane) {
         v = ld_u32(adj + p);
         if (v >= c.n_nodes) raise(c, 7, 0x92, qs, v);
         else {
-          u32 r = set_insert(seen, c.seen_cap, v);
+          u32 r = c.seen_bitmap ? bit_insert(seen, v) : set_insert(seen, c.seen_cap, v);
           if (r == 2) raise(c, 6, 0x93, qs, v);
           isnew = r == 1;
         }

@@ -46,7 +46,8 @@ __device__ bool recycle_slot(const Ctx &c, u32 qs, u32 lane) {
   if (nxt >= c.nq) return false;
   uint4 ff = make_uint4(kInvalidId, kInvalidId, kInvalidId, kInvalidId);
   uint4 *s4 = (uint4 *)(c.seen + (u64)qs * c.seen_cap);
-  for (u32 i = lane; i < c.seen_cap / 4; i += 32) __stcg(s4 + i, ff);
+  const uint4 sclear = c.seen_bitmap ? make_uint4(0, 0, 0, 0) : ff;
+  for (u32 i = lane; i < c.seen_cap / 4; i += 32) __stcg(s4 + i, sclear);
   uint4 *p4 = (uint4 *)(c.pset + (u64)qs * c.pset_cap);
   const uint4 pclear = c.pset_bitmap ? make_uint4(0, 0, 0, 0) : ff;
   for (u32 i = lane; i < c.pset_cap / 4; i += 32) __stcg(p4 + i, pclear);
@@ -120,7 +121,8 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut, u32 &lut_qid
     if (phase == PH_NEW) {
       const u32 qid = uld(&h->qid);
       if (lane == 0) {
-        set_insert(c.seen + (u64)qs * c.seen_cap, c.seen_cap, c.entry);
+        if (c.seen_bitmap) bit_insert(c.seen + (u64)qs * c.seen_cap, c.entry);
+        else set_insert(c.seen + (u64)qs * c.seen_cap, c.seen_cap, c.entry);
         st_u32(c.items + (u64)qs * c.WR, c.entry);
         st_u32(&h->n_items, 1); st_u32(&h->n_eval, 1); st_u32(&h->phase, PH_EVAL);
       }

@@ -329,10 +329,16 @@ int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W) {
   const u32 R = ix->desc.max_degree, WR = W * R;
   const u32 max_inflight = ix->tune.max_inflight ? ix->tune.max_inflight : 16384u;
   const u32 slots = nq < max_inflight ? nq : max_inflight;
-  const u32 seen_cap = ix->tune.visited_capacity ? ix->tune.visited_capacity : 32768u;
+  // exact visited set per query: a bitmap over the nodes when that is no larger than the hash set
+  // (one atomicOr, no probing, never full), else the hash set (config 5: 10M nodes)
+  u32 seen_cap = ix->tune.visited_capacity ? ix->tune.visited_capacity : 32768u;
+  const u32 hash_cap = seen_cap;
+  const u32 node_words = (u32)(((ix->desc.n_nodes + 31u) / 32u + 3u) & ~(u64)3u);
+  const bool seen_bitmap = node_words <= seen_cap;
+  if (seen_bitmap) seen_cap = node_words;
   // distinct-page set per query: a bitmap over the index's pages when that is smaller than the
   // hash set (config 3: 100,000 pages = 12.5 KB instead of 128 KB per query), else the hash set
-  u32 pset_cap = ix->desc.pq_m ? 4096u : seen_cap;
+  u32 pset_cap = ix->desc.pq_m ? 4096u : hash_cap;
   const u32 bitmap_words = ((ix->n_pages + 31u) / 32u + 3u) & ~3u;
   const bool pset_bitmap = bitmap_words <= pset_cap;
   if (pset_bitmap) pset_cap = bitmap_words;
@@ -374,7 +380,7 @@ int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W) {
   c.adjdeg = (u32 *)(b + o_adeg); c.pool = (u64 *)(b + o_pool);
   c.seen = (u32 *)(b + o_seen); c.pset = (u32 *)(b + o_pset);
   c.stash_tag = (u32 *)(b + o_stag); c.stash = (u32 *)(b + o_stash); c.stash_cap = stash_cap;
-  c.seen_cap = seen_cap; c.pset_cap = pset_cap; c.pset_bitmap = pset_bitmap ? 1u : 0u; c.n_qslots = slots;
+  c.seen_cap = seen_cap; c.pset_cap = pset_cap; c.pset_bitmap = pset_bitmap ? 1u : 0u; c.seen_bitmap = seen_bitmap ? 1u : 0u; c.n_qslots = slots;
   ix->qs_slots = slots; ix->qs_L = L; ix->qs_W = W; ix->qs_WR = WR; ix->qs_K = K;
   ix->qs_seen = seen_cap; ix->qs_pset = pset_cap; ix->qs_stash = ix->tune.stash_entries + 1u; ix->qs_nslots = ix->n_slots;
   ix->qs_units = ix->n_units;
@@ -600,7 +606,7 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   flush_wc();
   std::atomic_thread_fence(std::memory_order_seq_cst);
 
-  CK(cudaMemsetAsync(c.seen, 0xFF, (size_t)c.n_qslots * c.seen_cap * 4, stream));
+  CK(cudaMemsetAsync(c.seen, c.seen_bitmap ? 0x00 : 0xFF, (size_t)c.n_qslots * c.seen_cap * 4, stream));
   CK(cudaMemsetAsync(c.pset, c.pset_bitmap ? 0x00 : 0xFF, (size_t)c.n_qslots * c.pset_cap * 4, stream));
   if (c.stash_cap) CK(cudaMemsetAsync(c.stash_tag, 0xFF, (size_t)c.n_qslots * c.stash_cap * 4, stream));
   CK(launch_init(c, stream));

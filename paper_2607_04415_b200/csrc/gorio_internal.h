@@ -126,6 +126,7 @@ struct Ctx {
   u32 *stash_tag; // [n_qslots][stash_cap] node id of each stash entry (all ones = empty)
   u32 seen_cap, pset_cap, stash_cap;
   u32 pset_bitmap;   // 1: the page set is a bitmap over index pages (pset_cap words) instead of a hash set
+  u32 seen_bitmap;   // 1: the visited set is a bitmap over nodes (seen_cap words) instead of a hash set
   const void *queries;
   u32 *out_ids;
   void *out_dists;
