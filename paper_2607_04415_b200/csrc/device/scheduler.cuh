@@ -320,11 +320,13 @@ __device__ bool warp_ticket(int *count, u32 *head, u32 &idx, u32 lane) {
   return __shfl_sync(0xffffffffu, ok, 0) != 0u;
 }
 
-// Register budget: at most 80 per thread, so that 24 warps (61,440 registers) fit on an SM.  With
-// PQ navigation the per-warp table in shared memory allows 12 warps at most, so that variant is
-// built for 384 threads and may use twice the registers (no spills).
-template <bool PQ>
-__global__ void __launch_bounds__(PQ ? 384 : 768, 1) search_kernel(const Ctx c) {
+// Register budget: MAXT threads per block, one block per SM.  768 threads (24 warps, used when
+// the whole index is resident and there are many queries per SM) leave 80 registers per thread;
+// 512 threads (the default 16 warps whenever pages can be missed) leave 128 and need no spills.
+// With PQ navigation the per-warp table in shared memory allows 12 warps at most, so that
+// variant is built for 384 threads (168 registers).
+template <bool PQ, int MAXT>
+__global__ void __launch_bounds__(MAXT, 1) search_kernel(const Ctx c) {
   extern __shared__ u32 smem_lut[];
   const u32 lane = lane_id(), warp = threadIdx.x >> 5;
   if (blockIdx.x == 0 && warp == 0) { poller(c, lane); return; }

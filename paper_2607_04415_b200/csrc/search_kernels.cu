@@ -76,8 +76,9 @@ __global__ void cache_reset_kernel(const Ctx c, u32 preloaded) {
 cudaError_t preload_kernels() {
   cudaFuncAttributes a;
   cudaError_t e;
-  if ((e = cudaFuncGetAttributes(&a, search_kernel<false>)) != cudaSuccess) return e;
-  if ((e = cudaFuncGetAttributes(&a, search_kernel<true>)) != cudaSuccess) return e;
+  if ((e = cudaFuncGetAttributes(&a, search_kernel<false, 512>)) != cudaSuccess) return e;
+  if ((e = cudaFuncGetAttributes(&a, search_kernel<false, 768>)) != cudaSuccess) return e;
+  if ((e = cudaFuncGetAttributes(&a, search_kernel<true, 384>)) != cudaSuccess) return e;
   if ((e = cudaFuncGetAttributes(&a, init_kernel)) != cudaSuccess) return e;
   return cudaFuncGetAttributes(&a, cache_reset_kernel);
 }
@@ -97,21 +98,25 @@ static size_t search_smem(const Ctx &c, u32 warps) { return c.pq_m ? (size_t)war
 cudaError_t search_occupancy(u32 pq_m, u32 warps_per_block, int *blocks_per_sm) {
   if (pq_m) {
     const size_t smem = (size_t)warps_per_block * pq_m * kPqLutWords * 4;
-    cudaError_t e = cudaFuncSetAttribute(search_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(search_kernel<true, 384>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<true>, warps_per_block * 32, smem);
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<true, 384>, warps_per_block * 32, smem);
   }
-  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<false>, warps_per_block * 32, 0);
+  if (warps_per_block <= 16)
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<false, 512>, warps_per_block * 32, 0);
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<false, 768>, warps_per_block * 32, 0);
 }
 
 cudaError_t launch_search(const Ctx &c, u32 blocks, u32 warps_per_block, cudaStream_t s) {
   const size_t smem = search_smem(c, warps_per_block);
   if (c.pq_m) {
-    cudaError_t e = cudaFuncSetAttribute(search_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(search_kernel<true, 384>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    search_kernel<true><<<blocks, warps_per_block * 32, smem, s>>>(c);
+    search_kernel<true, 384><<<blocks, warps_per_block * 32, smem, s>>>(c);
+  } else if (warps_per_block <= 16) {
+    search_kernel<false, 512><<<blocks, warps_per_block * 32, 0, s>>>(c);
   } else {
-    search_kernel<false><<<blocks, warps_per_block * 32, 0, s>>>(c);
+    search_kernel<false, 768><<<blocks, warps_per_block * 32, 0, s>>>(c);
   }
   return cudaGetLastError();
 }
