@@ -60,7 +60,7 @@ __device__ __noinline__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
     if (pending) {
       node = ld_u32(items + j);
       page = unit_of(c, node);
-      w_first = ld_u64(c.ptab + page);    // in flight while the page set is probed
+      if (!c.identity) w_first = ld_u64(c.ptab + page);    // in flight while the page set is probed
       if (count_pages) {                  // distinct index pages, whatever the cache's unit
         const u32 ipage = node / c.npp;
         u32 r;
@@ -99,13 +99,19 @@ __device__ __noinline__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
     phase_mark(c, tq, S_I_SETUP, lane);
     for (u32 round = 0; __any_sync(0xffffffffu, pending); ++round) {
       u32 code = LK_NONE, slot = 0, gen = 0;
-      if (pending) code = page_lookup(c, page, qs * c.WR + j, round ? ld_u64(c.ptab + page) : w_first, slot, gen, st);
+      if (c.identity) {                   // whole index preloaded: unit u sits in slot u for good
+        if (pending) { code = LK_HIT; slot = page; }
+      } else if (pending) {
+        code = page_lookup(c, page, qs * c.WR + j, round ? ld_u64(c.ptab + page) : w_first, slot, gen, st);
+      }
       __syncwarp();
       phase_mark(c, tq, S_I_LOOKUP, lane);
       if (code == LK_WAIT) pending = false;
       const u32 hits = __ballot_sync(0xffffffffu, code == LK_HIT);
       if (hits) consume_group<PQ>(c, hits, qs, j, slot, phase, qid, node, worst, lane);
-      if (hits) {
+      if (hits && c.identity) {
+        if (code == LK_HIT) { st.hit++; n_done++; pending = false; }
+      } else if (hits) {
         __threadfence();
         if (code == LK_HIT) {
           // the bytes just read were the page's if its word still names this slot and fill
@@ -122,10 +128,10 @@ __device__ __noinline__ bool issue_batch(const Ctx &c, u32 qs, u32 lane) {
         }
       }
       phase_mark(c, tq, S_I_CONSUME, lane);
+      // (no stop check here: every round resolves its items or retries a bounded number of
+      // times, and run_query looks at the stop flag between phases)
       if (round > 1024) { if (lane == 0) raise(c, 8, 0x84, qs, base); break; }
-      if (warp_stopped(c)) break;
     }
-    if (warp_stopped(c)) break;
   }
 
 #pragma unroll

@@ -574,6 +574,8 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   c.vec128 = (ix->vec_bytes % 16 == 0 && ix->vec_bytes <= 384 && ((uintptr_t)queries_dev & 15) == 0) ? 1u : 0u;
   { const char *e = std::getenv("GORIO_CENSUS_MS"); c.census_ns = e ? (u64)std::atof(e) * 1000000ull : 0; }
   c.prof = std::getenv("GORIO_PROFILE") ? 1u : 0u;
+  // whole index preloaded page by page: slot p holds page p and no request can ever be posted
+  c.identity = (!ix->record_mode && ix->preloaded == ix->n_units && ix->n_slots == ix->n_units) ? 1u : 0u;
 
   // launch geometry: one block per SM by default
   const bool pq = d.pq_m != 0;
