@@ -31,7 +31,7 @@ METRIC = "QPS @ recall@10, 1M x 128 uint8, 20% cache, 20us miss"
 # dram__bytes_read.sum + dram__bytes_write.sum of one search_kernel launch on the default workload
 # (config 3, 10,000 queries, cold 20 % cache), mean of 8 launches of a single-pass ncu capture of this
 # very command; see profiles/search_kernel_cfg3_launch_list.md.  Reported only for that workload.
-NCU_DRAM_BYTES_PER_LAUNCH_CFG3 = 19.59e9 + 25.42e9
+NCU_DRAM_BYTES_PER_LAUNCH_CFG3 = 16.63e9 + 22.99e9
 PAPER_CONTEXT = ("paper (L40S + ConnectX-6 NVMe-oF, SIFT1M): G-ABaM 5650 QPS = 4.89x over blocking BaM, "
                  "G-Gust 1.31x over GustANN; context only, other hardware and transport")
 
