@@ -392,6 +392,110 @@ thread_local char g_global_error[256] = "";
 const char *kDeviceErr[] = {"", "", "", "", "", "device wait expired", "per-query capacity exhausted",
                             "corrupt index page", "internal state-machine check failed"};
 
+// Everything the kernels need for this search, gathered into the by-value context.
+void fill_ctx(gorio_index *ix, const void *queries_dev, u32 nq, u32 K, u32 L, u32 W, u32 *out_ids_dev, void *out_dists_dev,
+              u32 *out_pages_distinct_dev, u32 *out_counters_dev) {
+  const gorio_index_desc &d = ix->desc;
+  Ctx &c = ix->ctx;
+  c.n_nodes = (u32)d.n_nodes; c.dim = d.dim; c.dtype = d.dtype; c.R = d.max_degree; c.npp = d.nodes_per_page;
+  c.node_bytes = ix->node_bytes; c.vec_bytes = ix->vec_bytes; c.entry = d.entry_id; c.n_pages = ix->n_pages;
+  c.pq_m = d.pq_m; c.pq_dsub = d.pq_m ? d.dim / d.pq_m : 0; c.pq_cent = d.pq_centroids_dev; c.pq_codes = d.pq_codes_dev;
+  c.slot_data = ix->slot_data; c.ptab = ix->ptab; c.smeta = ix->smeta; c.parts = ix->parts; c.filled = ix->filled; c.cs = ix->cs;
+  c.n_slots = ix->n_slots; c.n_units = ix->n_units; c.slot_bytes = ix->slot_bytes; c.record_mode = ix->record_mode;
+  c.ring = ix->ring_d; c.ring_mask = ix->ring_cap - 1; c.ring_shift = ilog2(ix->ring_cap);
+  c.ring_dev = ix->ring_copy; c.host_ctl = ix->hctl_d;
+  c.fdone = ix->fdone_d; c.host_pages = ix->pages_dev;
+  c.ctl = ix->ctl;
+  u32 *qh = ix->ctl->q_heads;
+  int *cnt = ix->ctl->counts;
+  c.arr = Queue{(u32 *)ix->arr_buf, ix->arr_cap - 1, qh + 0, qh + 1, cnt + 2};
+  c.run = Queue{(u32 *)ix->run_buf, ix->runq_cap - 1, qh + 3, qh + 4, cnt + 3};
+  c.want = Queue{(u32 *)ix->want_buf, ix->want_cap - 1, qh + 6, qh + 7, cnt + 4};
+  c.nq = nq; c.K = K; c.L = L; c.W = W; c.WR = ix->qs_WR;
+  c.queries = queries_dev; c.out_ids = out_ids_dev; c.out_dists = out_dists_dev;
+  c.out_pages = out_pages_distinct_dev; c.out_counters = out_counters_dev;
+  c.timeout_ns = (u64)ix->cfg.timeout_ms * 1000000ull;
+  c.max_iters = 64u * L + 1024u;
+  c.blocking = ix->tune.blocking ? 1u : 0u;
+  c.idle_ns = 8000u;
+  // default backlog: 4 x the proxy's window, but no more than 1024 (about what keeps the host
+  // link busy) unless the window itself is larger
+  c.max_in_flight = ix->tune.request_backlog ? ix->tune.request_backlog
+                    : (4u * ix->cfg.max_outstanding < 1024u ? 4u * ix->cfg.max_outstanding : 1024u);
+  if (c.max_in_flight < ix->cfg.max_outstanding) c.max_in_flight = ix->cfg.max_outstanding;
+  c.vec128 = (ix->vec_bytes % 16 == 0 && ix->vec_bytes <= 384 && ((uintptr_t)queries_dev & 15) == 0) ? 1u : 0u;
+  { const char *e = std::getenv("GORIO_CENSUS_MS"); c.census_ns = e ? (u64)std::atof(e) * 1000000ull : 0; }
+  c.prof = std::getenv("GORIO_PROFILE") ? 1u : 0u;
+  // whole index preloaded page by page: slot p holds page p and no request can ever be posted
+  c.identity = (!ix->record_mode && ix->preloaded == ix->n_units && ix->n_slots == ix->n_units) ? 1u : 0u;
+}
+
+// Launch geometry of the persistent kernel: blocks and warps per block.
+int launch_geometry(gorio_index *ix, u32 nq, u32 *blocks_out, u32 *warps_out) {
+  const gorio_index_desc &d = ix->desc;
+  // launch geometry: one block per SM by default
+  const bool pq = d.pq_m != 0;
+  // default warps per SM: 16 when pages will be missed (more warps lengthen every copy and arrival);
+  // with every page resident one warp carries one query at a time, so no more than there are
+  // queries per SM (fewer idle warps polling the queues), within 8..24
+  u32 auto_warps = 16u;
+  if (ix->n_slots >= ix->n_units) {
+    auto_warps = (nq + (u32)ix->n_sms - 1) / (u32)ix->n_sms;
+    auto_warps = auto_warps < 8u ? 8u : (auto_warps > 24u ? 24u : auto_warps);
+  }
+  u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 10u : auto_warps);
+  if (pq) {      // one table per warp in shared memory; the PQ kernel is built for at most 12 warps
+    u32 lim = (220u * 1024u) / (d.pq_m * kPqLutWords * 4u);
+    if (lim > 12u) lim = 12u;
+    if (warps > lim) warps = lim;
+  }
+  if (warps < 2) return fail(ix, GORIO_ERR_INVALID_ARG, "search: need at least 2 warps per block (the poller and a worker)");
+  int occ = 0;
+  CK(search_occupancy(d.pq_m, warps, &occ));
+  if (occ < 1) return fail(ix, GORIO_ERR_INVALID_ARG, "search: launch geometry does not fit an SM");
+  u32 bps = ix->tune.blocks_per_sm ? ix->tune.blocks_per_sm : 1u;
+  if ((int)bps > occ) bps = (u32)occ;
+  *blocks_out = (u32)ix->n_sms * bps;
+  *warps_out = warps;
+  return GORIO_OK;
+}
+
+// Debug aids (GORIO_CENSUS_MS, GORIO_PROFILE): print what the kernel recorded.
+void print_diagnostics(const Ctx &c, const Ctl &h) {
+  if (c.census_ns)
+    std::fprintf(stderr, "[gorio census] slots: unused %u, changing owner %u, FILLING %u, ARRIVED %u, RESIDENT ref %u, RESIDENT noref %u | "
+                 "pages WANTED %u | queries awaiting %u (items %u) | queues want %d arr %d run %d | done %u posted %u\n",
+                 h.census[0], h.census[1], h.census[2], h.census[3], h.census[4], h.census[5], h.census[6], h.census[7],
+                 h.census[8], (int)h.census[9], (int)h.census[10], (int)h.census[11], h.census[12], h.census[13]);
+  if (c.prof) {
+    const char *names[] = {"merge", "issue_eval", "issue_expand", "collect", "pool", "lut", "adc", "finish", "recycle",
+                           "(issue: setup", "lookup", "consume", "tail)"};
+    std::fprintf(stderr, "[gorio profile] warp ms per query step (cumulative since stats_reset):");
+    for (int i = 0; i < 13; ++i) std::fprintf(stderr, " %s %.1f", names[i], h.stats[S_P_MERGE + i] / 1e6);
+    std::fprintf(stderr, " | control reads %llu | copies: loads issued -> bytes arrived %.1f",
+                 (unsigned long long)h.stats[S_POLLS], h.stats[S_C_DATA] / 1e6);
+    std::fprintf(stderr, " | arrival: head %.1f walk %.1f group %.1f complete %.1f finish %.1f", h.stats[S_A_HEAD] / 1e6,
+                 h.stats[S_A_WALK] / 1e6, h.stats[S_A_GROUP] / 1e6, h.stats[S_A_COMPLETE] / 1e6, h.stats[S_A_FINISH] / 1e6);
+    std::fprintf(stderr, " | arrivals %.1f copies %.1f queries %.1f idle %.1f\n", h.stats[S_T_ARR] / 1e6, h.stats[S_T_CPY] / 1e6,
+                 h.stats[S_T_RUN] / 1e6, h.stats[S_T_IDLE] / 1e6);
+  }
+}
+
+// The search did not end cleanly: status and a message with the site code and queue / proxy progress.
+int device_failure(gorio_index *ix, const Ctl &h, u32 nq) {
+  char buf[640];
+  const u32 s = h.status ? h.status : (u32)GORIO_ERR_INTERNAL;
+  std::snprintf(buf, sizeof buf,
+                "device: %s (site 0x%x, %u, %u, %u; block %u thread %u; done %u/%u; posted %u; arrivals %u/%u; "
+                "runnable %u/%u; want %u/%u; proxy consumed %u published %u outstanding %u queued %u "
+                "[head command %u ack %u])",
+                s < 9 ? kDeviceErr[s] : "?", h.dbg[0], h.dbg[1], h.dbg[2], h.dbg[3], h.dbg[4], h.dbg[5], h.done, nq,
+                h.ring_head, h.q_heads[0], h.q_heads[1], h.q_heads[3], h.q_heads[4], h.q_heads[6], h.q_heads[7],
+                ix->px_dbg[0], ix->px_dbg[1], ix->px_dbg[2], ix->px_dbg[3], ix->px_dbg[4], ix->px_dbg[5]);
+  return fail(ix, (int)s, buf);
+}
+
+
 }  // namespace
 
 namespace gorio {
@@ -543,63 +647,11 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   int st = ensure_qstate(ix, nq, K, L, W);
   if (st != GORIO_OK) return st;
 
-  const gorio_index_desc &d = ix->desc;
+  fill_ctx(ix, queries_dev, nq, K, L, W, out_ids_dev, out_dists_dev, out_pages_distinct_dev, out_counters_dev);
   Ctx &c = ix->ctx;
-  c.n_nodes = (u32)d.n_nodes; c.dim = d.dim; c.dtype = d.dtype; c.R = d.max_degree; c.npp = d.nodes_per_page;
-  c.node_bytes = ix->node_bytes; c.vec_bytes = ix->vec_bytes; c.entry = d.entry_id; c.n_pages = ix->n_pages;
-  c.pq_m = d.pq_m; c.pq_dsub = d.pq_m ? d.dim / d.pq_m : 0; c.pq_cent = d.pq_centroids_dev; c.pq_codes = d.pq_codes_dev;
-  c.slot_data = ix->slot_data; c.ptab = ix->ptab; c.smeta = ix->smeta; c.parts = ix->parts; c.filled = ix->filled; c.cs = ix->cs;
-  c.n_slots = ix->n_slots; c.n_units = ix->n_units; c.slot_bytes = ix->slot_bytes; c.record_mode = ix->record_mode;
-  c.ring = ix->ring_d; c.ring_mask = ix->ring_cap - 1; c.ring_shift = ilog2(ix->ring_cap);
-  c.ring_dev = ix->ring_copy; c.host_ctl = ix->hctl_d;
-  c.fdone = ix->fdone_d; c.host_pages = ix->pages_dev;
-  c.ctl = ix->ctl;
-  u32 *qh = ix->ctl->q_heads;
-  int *cnt = ix->ctl->counts;
-  c.arr = Queue{(u32 *)ix->arr_buf, ix->arr_cap - 1, qh + 0, qh + 1, cnt + 2};
-  c.run = Queue{(u32 *)ix->run_buf, ix->runq_cap - 1, qh + 3, qh + 4, cnt + 3};
-  c.want = Queue{(u32 *)ix->want_buf, ix->want_cap - 1, qh + 6, qh + 7, cnt + 4};
-  c.nq = nq; c.K = K; c.L = L; c.W = W; c.WR = ix->qs_WR;
-  c.queries = queries_dev; c.out_ids = out_ids_dev; c.out_dists = out_dists_dev;
-  c.out_pages = out_pages_distinct_dev; c.out_counters = out_counters_dev;
-  c.timeout_ns = (u64)ix->cfg.timeout_ms * 1000000ull;
-  c.max_iters = 64u * L + 1024u;
-  c.blocking = ix->tune.blocking ? 1u : 0u;
-  c.idle_ns = 8000u;
-  // default backlog: 4 x the proxy's window, but no more than 1024 (about what keeps the host
-  // link busy) unless the window itself is larger
-  c.max_in_flight = ix->tune.request_backlog ? ix->tune.request_backlog
-                    : (4u * ix->cfg.max_outstanding < 1024u ? 4u * ix->cfg.max_outstanding : 1024u);
-  if (c.max_in_flight < ix->cfg.max_outstanding) c.max_in_flight = ix->cfg.max_outstanding;
-  c.vec128 = (ix->vec_bytes % 16 == 0 && ix->vec_bytes <= 384 && ((uintptr_t)queries_dev & 15) == 0) ? 1u : 0u;
-  { const char *e = std::getenv("GORIO_CENSUS_MS"); c.census_ns = e ? (u64)std::atof(e) * 1000000ull : 0; }
-  c.prof = std::getenv("GORIO_PROFILE") ? 1u : 0u;
-  // whole index preloaded page by page: slot p holds page p and no request can ever be posted
-  c.identity = (!ix->record_mode && ix->preloaded == ix->n_units && ix->n_slots == ix->n_units) ? 1u : 0u;
-
-  // launch geometry: one block per SM by default
-  const bool pq = d.pq_m != 0;
-  // default warps per SM: 16 when pages will be missed (more warps lengthen every copy and arrival);
-  // with every page resident one warp carries one query at a time, so no more than there are
-  // queries per SM (fewer idle warps polling the queues), within 8..24
-  u32 auto_warps = 16u;
-  if (ix->n_slots >= ix->n_units) {
-    auto_warps = (nq + (u32)ix->n_sms - 1) / (u32)ix->n_sms;
-    auto_warps = auto_warps < 8u ? 8u : (auto_warps > 24u ? 24u : auto_warps);
-  }
-  u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 10u : auto_warps);
-  if (pq) {      // one table per warp in shared memory; the PQ kernel is built for at most 12 warps
-    u32 lim = (220u * 1024u) / (d.pq_m * kPqLutWords * 4u);
-    if (lim > 12u) lim = 12u;
-    if (warps > lim) warps = lim;
-  }
-  if (warps < 2) return fail(ix, GORIO_ERR_INVALID_ARG, "search: need at least 2 warps per block (the poller and a worker)");
-  int occ = 0;
-  CK(search_occupancy(d.pq_m, warps, &occ));
-  if (occ < 1) return fail(ix, GORIO_ERR_INVALID_ARG, "search: launch geometry does not fit an SM");
-  u32 bps = ix->tune.blocks_per_sm ? ix->tune.blocks_per_sm : 1u;
-  if ((int)bps > occ) bps = (u32)occ;
-  const u32 blocks = (u32)ix->n_sms * bps;
+  u32 blocks = 0, warps = 0;
+  st = launch_geometry(ix, nq, &blocks, &warps);
+  if (st != GORIO_OK) return st;
 
   // reset the host-visible rings while the proxy is idle
   std::memset(ix->ring_h, 0, (size_t)ix->ring_cap * 8);
@@ -633,36 +685,9 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   CK(cudaMemcpyAsync(&h, ix->ctl, sizeof(Ctl), cudaMemcpyDeviceToHost, stream));
   CK(cudaStreamSynchronize(stream));
   ix->host_search_ns += (u64)std::chrono::duration_cast<std::chrono::nanoseconds>(Clock::now() - t_begin).count();
-  if (c.census_ns)
-    std::fprintf(stderr, "[gorio census] slots: unused %u, changing owner %u, FILLING %u, ARRIVED %u, RESIDENT ref %u, RESIDENT noref %u | "
-                 "pages WANTED %u | queries awaiting %u (items %u) | queues want %d arr %d run %d | done %u posted %u\n",
-                 h.census[0], h.census[1], h.census[2], h.census[3], h.census[4], h.census[5], h.census[6], h.census[7],
-                 h.census[8], (int)h.census[9], (int)h.census[10], (int)h.census[11], h.census[12], h.census[13]);
-  if (c.prof) {
-    const char *names[] = {"merge", "issue_eval", "issue_expand", "collect", "pool", "lut", "adc", "finish", "recycle",
-                           "(issue: setup", "lookup", "consume", "tail)"};
-    std::fprintf(stderr, "[gorio profile] warp ms per query step (cumulative since stats_reset):");
-    for (int i = 0; i < 13; ++i) std::fprintf(stderr, " %s %.1f", names[i], h.stats[S_P_MERGE + i] / 1e6);
-    std::fprintf(stderr, " | control reads %llu | copies: loads issued -> bytes arrived %.1f",
-                 (unsigned long long)h.stats[S_POLLS], h.stats[S_C_DATA] / 1e6);
-    std::fprintf(stderr, " | arrival: head %.1f walk %.1f group %.1f complete %.1f finish %.1f", h.stats[S_A_HEAD] / 1e6,
-                 h.stats[S_A_WALK] / 1e6, h.stats[S_A_GROUP] / 1e6, h.stats[S_A_COMPLETE] / 1e6, h.stats[S_A_FINISH] / 1e6);
-    std::fprintf(stderr, " | arrivals %.1f copies %.1f queries %.1f idle %.1f\n", h.stats[S_T_ARR] / 1e6, h.stats[S_T_CPY] / 1e6,
-                 h.stats[S_T_RUN] / 1e6, h.stats[S_T_IDLE] / 1e6);
-  }
+  print_diagnostics(c, h);
   if (ix->px_error.load()) return fail(ix, GORIO_ERR_INTERNAL, "proxy: descriptor out of range");
-  if (h.status != 0 || h.stop != 1) {
-    char buf[640];
-    const u32 s = h.status ? h.status : (u32)GORIO_ERR_INTERNAL;
-    std::snprintf(buf, sizeof buf,
-                  "device: %s (site 0x%x, %u, %u, %u; block %u thread %u; done %u/%u; posted %u; arrivals %u/%u; "
-                  "runnable %u/%u; want %u/%u; proxy consumed %u published %u outstanding %u queued %u "
-                  "[head command %u ack %u])",
-                  s < 9 ? kDeviceErr[s] : "?", h.dbg[0], h.dbg[1], h.dbg[2], h.dbg[3], h.dbg[4], h.dbg[5], h.done, nq,
-                  h.ring_head, h.q_heads[0], h.q_heads[1], h.q_heads[3], h.q_heads[4], h.q_heads[6], h.q_heads[7],
-                  ix->px_dbg[0], ix->px_dbg[1], ix->px_dbg[2], ix->px_dbg[3], ix->px_dbg[4], ix->px_dbg[5]);
-    return fail(ix, (int)s, buf);
-  }
+  if (h.status != 0 || h.stop != 1) return device_failure(ix, h, nq);
   ix->cache_dirty = false;
   return GORIO_OK;
 }
