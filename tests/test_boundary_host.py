@@ -109,3 +109,23 @@ def test_two_rank_gloo_gather_restores_global_order():
         assert p.exitcode == 0
     assert full == [[i, 10 * i] for i in range(nq)]
     assert tmax == 2.0
+
+
+def test_bench_reference_arm_prints_the_contract_line_on_cpu():
+    """`bench.py --impl reference` times the oracle and needs no GPU: one JSON line with the
+    contract's keys, on a shrunken workload so that the CPU suite stays short."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference", "--config", "3",
+                          "--scale", "0.01", "--nq", "64", "--steps", "1", "--warmup", "1"],
+                         capture_output=True, text=True, timeout=300, cwd=root)
+    assert out.returncode == 0, out.stderr[-800:]
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    for key in ("impl", "metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better",
+                "scaling", "vs_baseline", "dtype", "data", "config", "cpu_baseline", "e2e"):
+        assert key in line, key
+    assert line["impl"] == "reference" and line["value"] > 0 and line["vs_baseline"] is None
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
