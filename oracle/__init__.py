@@ -38,7 +38,9 @@ class _OrcIndex(ctypes.Structure):
 def build(force: bool = False) -> str:
     """Compile beam_oracle.c with gcc into a shared library next to it."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        subprocess.check_call(["gcc", "-O2", "-std=c11", "-shared", "-fPIC", "-o", _LIB, _SRC])
+        tmp = f"{_LIB}.{os.getpid()}.tmp"      # several processes may find it stale at once: never a half-written file
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-shared", "-fPIC", "-o", tmp, _SRC])
+        os.replace(tmp, _LIB)
     return _LIB
 
 

@@ -5,9 +5,9 @@
  * Only tests, the smoke check and the benchmark's cpu_baseline leg may build or call
  * it; the product path never does, and the two share no code.
  *
- * What it computes.  The paper (Section 2.2) describes graph ANNS as a loop that
- * "expands graph nodes, evaluates vector distances, updates candidate queues and
- * discovers the next pages to fetch" on a DiskANN-style index (Section 5.1) and
+ * What it computes.  The paper (Section 2.2) describes graph ANNS only as a loop of
+ * four activities -- node expansion, distance evaluation, candidate-queue update and
+ * discovery of the pages needed next -- on a DiskANN-style index (Section 5.1) and
  * gives no further definition.  The reading implemented here is the standard
  * best-first beam search of width W over a bounded sorted list of size L:
  *

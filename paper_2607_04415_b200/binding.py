@@ -39,7 +39,7 @@ class _CacheCfg(ctypes.Structure):
     _fields_ = [("capacity_pages", ctypes.c_uint64), ("remote_latency_ns", ctypes.c_uint32),
                 ("max_outstanding", ctypes.c_uint32), ("preload", ctypes.c_uint32),
                 ("timeout_ms", ctypes.c_uint32), ("granularity", ctypes.c_uint32),
-                ("reserved1", ctypes.c_uint32)]
+                ("copy_mode", ctypes.c_uint32)]
 
 
 class _Tuning(ctypes.Structure):
@@ -99,6 +99,48 @@ def load_library():
     return lib
 
 
+def _invalid(msg):
+    return GorioError(1, msg)
+
+
+def check_queries(queries, dim: int, dtype: str, device_index: Optional[int] = None):
+    """Shape, element type, layout and placement of a query tensor, checked before its raw
+    pointer goes to the library (which cannot see any of them): [nq, dim], uint8 or float32 as
+    the index, contiguous, on the index's CUDA device."""
+    want = torch.uint8 if dtype == "u8" else torch.float32
+    if not isinstance(queries, torch.Tensor) or queries.dim() != 2:
+        raise _invalid("queries must be a 2-D torch tensor [nq, dim]")
+    if queries.shape[1] != dim:
+        raise _invalid(f"queries have {queries.shape[1]} columns, the index has dim {dim}")
+    if queries.dtype != want:
+        raise _invalid(f"queries are {queries.dtype}, the index holds {want}")
+    if not queries.is_contiguous():
+        raise _invalid("queries must be contiguous (row major)")
+    if not queries.is_cuda:
+        raise _invalid("queries must be a CUDA tensor")
+    if device_index is not None and queries.device.index != device_index:
+        raise _invalid(f"queries live on cuda:{queries.device.index}, the index on cuda:{device_index}")
+    if queries.data_ptr() % 4 != 0:
+        raise _invalid("queries must be at least 4-byte aligned")
+
+
+def check_resident_pages(pages_dev, n_nodes: int, nodes_per_page: int, device):
+    """The device page store handed to the allocation-free entry: uint8, contiguous, on the
+    queries' device, at least 4-byte aligned and large enough for every page the index
+    description implies (the kernels read the page of any neighbour id below n_nodes)."""
+    if nodes_per_page < 1 or n_nodes < 1:
+        raise _invalid("n_nodes and nodes_per_page must be positive")
+    n_pages = (n_nodes + nodes_per_page - 1) // nodes_per_page
+    if not isinstance(pages_dev, torch.Tensor) or pages_dev.dtype != torch.uint8 or not pages_dev.is_contiguous():
+        raise _invalid("pages_dev must be a contiguous uint8 torch tensor")
+    if not pages_dev.is_cuda or pages_dev.device != device:
+        raise _invalid("pages_dev must live on the same CUDA device as the queries")
+    if pages_dev.numel() < n_pages * 4096:
+        raise _invalid(f"pages_dev holds {pages_dev.numel()} bytes, the index description needs {n_pages * 4096}")
+    if pages_dev.data_ptr() % 4 != 0:
+        raise _invalid("pages_dev must be at least 4-byte aligned")
+
+
 class Index:
     """gorio_index_open / cache_config / search / stats / close with torch tensors for memory."""
 
@@ -146,11 +188,13 @@ class Index:
             raise GorioError(status, detail or self._lib.gorio_status_str(status).decode())
 
     def cache_config(self, capacity_pages, remote_latency_ns=0, max_outstanding=256, preload=False,
-                     timeout_ms=0, granularity="page"):
-        """granularity: "page" (a miss fetches the 4 KB page) or "record" (only the wanted node's record)."""
+                     timeout_ms=0, granularity="page", copy_engine=False):
+        """granularity: "page" (a miss fetches the 4 KB page) or "record" (only the wanted node's record).
+        copy_engine: the proxy thread copies each page itself (one cudaMemcpyAsync per request)
+        instead of commanding warps of the search kernel to pull it."""
         gran = {"page": 0, "record": 1}[granularity]
         cfg = _CacheCfg(int(capacity_pages), int(remote_latency_ns), int(max_outstanding), int(bool(preload)),
-                        int(timeout_ms), gran, 0)
+                        int(timeout_ms), gran, 1 if copy_engine else 0)
         self._check(self._lib.gorio_cache_config(self._h, ctypes.byref(cfg)))
 
     def set_tuning(self, max_inflight=0, visited_capacity=0, warps_per_block=0, blocks_per_sm=0, stash_entries=0,
@@ -161,7 +205,7 @@ class Index:
 
     def search(self, queries: torch.Tensor, K: int, L: int, W: int, want_counters=True, stream=None):
         """queries: CUDA tensor [nq, dim] of the index dtype.  Returns dict of CUDA tensors."""
-        assert queries.is_cuda and queries.is_contiguous()
+        check_queries(queries, self.dim, self.dtype, self.device)
         nq = queries.shape[0]
         dev = queries.device
         ids = torch.empty((nq, K), dtype=torch.int32, device=dev)
@@ -178,6 +222,8 @@ class Index:
         """Host buffers in, host buffers out (the copies happen inside the C call).  `out` may
         supply preallocated (e.g. pinned) arrays: ids, dists, pages, counters."""
         q = np.ascontiguousarray(queries)
+        if q.ndim != 2 or q.shape[1] != self.dim or q.dtype != (np.uint8 if self.dtype == "u8" else np.float32):
+            raise _invalid(f"queries must be [nq, {self.dim}] of the index's element type")
         nq = q.shape[0]
         out = out or {}
         ids = out.get("ids", np.empty((nq, K), dtype=np.uint32))
@@ -217,9 +263,9 @@ def search_resident_noalloc(pages_dev: torch.Tensor, n_nodes: int, dim: int, dty
     caller's allocator, before the call).  For callers that cannot call cudaMalloc; limits
     and sharing rules are in include/gorio.h."""
     lib = load_library()
-    assert pages_dev.is_cuda and pages_dev.dtype == torch.uint8 and pages_dev.is_contiguous()
-    assert queries.is_cuda and queries.is_contiguous()
     u8 = str(dtype) in ("u8", "uint8")
+    check_queries(queries, dim, "u8" if u8 else "f32")
+    check_resident_pages(pages_dev, n_nodes, nodes_per_page, queries.device)
     d = _IndexDesc()
     d.n_nodes, d.dim, d.dtype = n_nodes, dim, 0 if u8 else 1
     d.max_degree, d.nodes_per_page, d.page_bytes, d.entry_id = max_degree, nodes_per_page, 4096, entry_id

@@ -28,6 +28,18 @@ def _source_hash() -> str:
     return h.hexdigest()
 
 
+def kernel_source_hash() -> str:
+    """Hash of the device code alone (kernels and the structures they share with the host):
+    what a profiler capture of a kernel's memory traffic is tied to.  Host-side edits do not
+    change it."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in ["search_kernels.cu", "gorio_internal.h"] + [x for x in HEADERS if x.startswith("device")]:
+        with open(os.path.join(CSRC, f), "rb") as fh:
+            h.update(f.encode() + b"\0" + fh.read())
+    return h.hexdigest()[:16]
+
+
 def _stale() -> bool:
     """True unless the library was built from exactly these sources (file times do not survive a
     copy of the tree to another machine, contents do)."""

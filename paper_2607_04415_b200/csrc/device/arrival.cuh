@@ -93,9 +93,10 @@ __device__ void consume_arrival(const Ctx &c, u32 v, u32 lane) {
   const u32 page = sm_page(m), gen = sm_gen(m);
   if (page >= c.n_units) { if (lane == 0) raise(c, 8, 0x76, slot, page); return; }
   u32 head = 0, bad = 0;
-  if (lane == 0) {
+  if (lane == 0 && !c.dma_fill) {
     // acquire the copier's stores into the slot (normally long done: the completion was
-    // published at least the remote latency after the bytes arrived)
+    // published at least the remote latency after the bytes arrived).  With copy-engine
+    // fills the proxy publishes only after the copy has completed, so there is nothing to wait for.
     u32 spins = 0;
     while (ld_u32(c.filled + slot) != gen) {
       __nanosleep(100);

@@ -93,8 +93,8 @@ __device__ void idle_step(const Ctx &c, u32 lane) {
   __syncwarp();
 }
 
-// Blocking mode (the demand-paging baseline the paper compares against, Section 5.1: misses
-// "issue remote reads and wait for page readiness"): the warp keeps its query and waits in
+// Blocking mode (the demand-paging baseline the paper compares against, Section 5.1, in which
+// a miss starts the remote read and the requester stays put until the page is there): the warp keeps its query and waits in
 // place until the batch it issued is complete.  It still moves pages while it waits -- someone
 // has to -- but it never picks up another query, so at most one query per warp is in flight.
 template <bool PQ>

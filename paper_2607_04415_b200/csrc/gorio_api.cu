@@ -1,7 +1,7 @@
 // Host side of the C ABI declared in include/gorio.h: resource management, the blocking
 // search call, and the CPU proxy thread that services page requests from the emulated
-// remote tier (paper Section 3.3: the proxy "batches submissions and completions, controls
-// outstanding remote I/O, and publishes ready state", and never looks at search state).
+// remote tier (paper Section 3.3: the proxy groups submissions and completions, bounds the
+// remote reads in flight and makes arrivals visible to the GPU; it never looks at search state).
 #include <atomic>
 #if defined(__x86_64__) || defined(__i386__)
 #include <immintrin.h>
@@ -31,6 +31,9 @@ inline u32 next_pow2(u64 v) { u32 p = 1; while (p < v) p <<= 1; return p; }
 inline u32 ilog2(u32 v) { u32 s = 0; while ((1u << s) < v) ++s; return s; }
 
 enum ProxyState : int { PX_IDLE = 0, PX_RUN = 1, PX_EXIT = 2 };
+constexpr int kFillStreams = 4;
+constexpr int kFillEvents = 256;
+constexpr u32 kFillBatch = 32;      // most copies the proxy issues before it looks at completions again
 
 }  // namespace
 
@@ -82,6 +85,10 @@ struct gorio_index {
   std::atomic<int> px_error{0};
   cudaStream_t own_stream = nullptr;
   cudaEvent_t done_ev = nullptr;
+  // copy-engine mode of the proxy: streams the proxy issues its page copies on, and a ring of
+  // events through which it learns that a batch of copies has landed
+  cudaStream_t fill_streams[kFillStreams] = {};
+  cudaEvent_t fill_events[kFillEvents] = {};
 
   // statistics
   u64 host_fetched_bytes = 0;
@@ -155,7 +162,7 @@ void free_qstate(gorio_index *ix) {
 // It issues no CUDA calls while a search runs: commands, acknowledgements and completions
 // all travel through host-mapped memory.
 // ---------------------------------------------------------------------------------------
-struct InService { u32 slot; u32 idx; Clock::time_point admitted; };
+struct InService { u32 slot; u32 idx; Clock::time_point admitted; u64 ev; };
 
 void proxy_service(gorio_index *ix) {
   const u32 ring_mask = ix->ring_cap - 1, ring_shift = ilog2(ix->ring_cap);
@@ -165,6 +172,13 @@ void proxy_service(gorio_index *ix) {
   volatile u32 *hctl = ix->hctl_h;
   volatile u32 *fdone = ix->fdone_h;
   u32 tail = 0, ct = 0, outstanding = 0;
+  // copy-engine mode (gorio_cache_cfg.copy_mode): the proxy itself moves each page with one
+  // cudaMemcpyAsync from the pinned store into the slot, on a few streams of its own, and learns
+  // that a batch has landed by querying an event recorded behind it -- no kernel takes part in a
+  // fill, so nothing needs a free block slot next to the persistent kernel.
+  const bool dma = ix->cfg.copy_mode == GORIO_COPY_ENGINE;
+  u64 ev_head = 0, ev_tail = 0;       // events recorded / events known complete (sequence numbers)
+  int fill_k = 0;
   std::deque<InService> inflight;
   u64 fetched = 0, max_seen = 0, batches = 0;
   u64 service_ns = 0, ack_wait_iters = 0, window_full_iters = 0, ring_empty_iters = 0, iters = 0, out_sum = 0;
@@ -187,7 +201,8 @@ void proxy_service(gorio_index *ix) {
     // 1. admit descriptors while the in-service window has room; each becomes a copy command
     u32 admitted = 0;
     const Clock::time_point now0 = Clock::now();
-    while (outstanding < max_out) {
+    const bool ev_room = !dma || ev_head - ev_tail < (u64)kFillEvents;
+    while (outstanding < max_out && ev_room && (!dma || admitted < kFillBatch)) {
       const u64 e = ring[tail & ring_mask];
       const u32 lap = ((tail >> ring_shift) % 255u) + 1u;
       if ((u32)(e & 0xFFu) != lap) break;
@@ -196,14 +211,46 @@ void proxy_service(gorio_index *ix) {
         ix->px_error.store(1);   // a descriptor the GPU could not have produced
         return;
       }
-      inflight.push_back({slot, tail, now0});
+      if (dma) {
+        // the page, or at record granularity the 16-byte-aligned span that covers the record
+        const u8 *src = (const u8 *)ix->desc.host_pages + (size_t)page * kPageBytes;
+        size_t bytes = kPageBytes;
+        if (ix->record_mode) {
+          const u32 npp = ix->desc.nodes_per_page, off = (page % npp) * ix->node_bytes;
+          src = (const u8 *)ix->desc.host_pages + (size_t)(page / npp) * kPageBytes + (off & ~15u);
+          bytes = (size_t)(((off & 15u) + ix->node_bytes + 15u) >> 4) * 16u;
+        }
+        if (cudaMemcpyAsync(ix->slot_data + (size_t)slot * ix->slot_bytes, src, bytes, cudaMemcpyHostToDevice,
+                            ix->fill_streams[fill_k]) != cudaSuccess) {
+          ix->px_error.store(2);
+          return;
+        }
+      }
+      inflight.push_back({slot, tail, now0, ev_head});
       ++tail; ++outstanding; ++admitted;
     }
     if (admitted) {
-      hctl[2] = tail;                             // requests [0, tail) may be copied now
-      flush_wc();
+      if (dma) {
+        if (cudaEventRecord(ix->fill_events[ev_head % kFillEvents], ix->fill_streams[fill_k]) != cudaSuccess) {
+          ix->px_error.store(2);
+          return;
+        }
+        ++ev_head;
+        fill_k = (fill_k + 1) % kFillStreams;
+      } else {
+        hctl[2] = tail;                           // requests [0, tail) may be copied now
+        flush_wc();
+      }
       ++batches;
       if (outstanding > max_seen) max_seen = outstanding;
+    }
+    if (dma) {                                    // which batches have landed (events complete in any order across streams)
+      while (ev_tail < ev_head) {
+        const cudaError_t qe = cudaEventQuery(ix->fill_events[ev_tail % kFillEvents]);
+        if (qe == cudaErrorNotReady) break;
+        if (qe != cudaSuccess) { ix->px_error.store(2); return; }
+        ++ev_tail;
+      }
     }
     if (outstanding >= max_out) {
       if ((u32)(ring[tail & ring_mask] & 0xFFu) == ((tail >> ring_shift) % 255u) + 1u) ++window_full_iters;
@@ -217,7 +264,8 @@ void proxy_service(gorio_index *ix) {
       while (!inflight.empty()) {
         const InService &r = inflight.front();
         if (now - r.admitted < latency) break;
-        if ((fdone[r.idx & ring_mask] & 0xFFu) != ((r.idx >> ring_shift) % 255u) + 1u) { ++ack_wait_iters; break; }
+        if (dma ? r.ev >= ev_tail
+                : (fdone[r.idx & ring_mask] & 0xFFu) != ((r.idx >> ring_shift) % 255u) + 1u) { ++ack_wait_iters; break; }
         service_ns += (u64)std::chrono::duration_cast<std::chrono::nanoseconds>(now - r.admitted).count();
         ++ct; ++published;
         inflight.pop_front();
@@ -230,6 +278,8 @@ void proxy_service(gorio_index *ix) {
       }
     }
   }
+  if (dma)       // nothing of this search may still be in flight when the caller frees or re-creates the cache
+    for (int i = 0; i < kFillStreams; ++i) cudaStreamSynchronize(ix->fill_streams[i]);
   if (trace) {
     std::fprintf(stderr, "[gorio proxy] per 10 ms: fetched(k)/mean outstanding:");
     u64 prev = 0;
@@ -427,6 +477,7 @@ void fill_ctx(gorio_index *ix, const void *queries_dev, u32 nq, u32 K, u32 L, u3
   { const char *e = std::getenv("GORIO_CENSUS_MS"); c.census_ns = e ? (u64)std::atof(e) * 1000000ull : 0; }
   c.prof = std::getenv("GORIO_PROFILE") ? 1u : 0u;
   // whole index preloaded page by page: slot p holds page p and no request can ever be posted
+  c.dma_fill = ix->cfg.copy_mode == GORIO_COPY_ENGINE ? 1u : 0u;
   c.identity = (!ix->record_mode && ix->preloaded == ix->n_units && ix->n_slots == ix->n_units) ? 1u : 0u;
 }
 
@@ -566,6 +617,10 @@ int gorio_index_open(const gorio_index_desc *d, int cuda_device, gorio_index **o
   cudaMemset(ix->ctl, 0, sizeof(Ctl));
   if (cudaStreamCreateWithFlags(&ix->own_stream, cudaStreamNonBlocking) != cudaSuccess) return bail(GORIO_ERR_CUDA);
   if (cudaEventCreateWithFlags(&ix->done_ev, cudaEventDisableTiming) != cudaSuccess) return bail(GORIO_ERR_CUDA);
+  for (int i = 0; i < kFillStreams; ++i)
+    if (cudaStreamCreateWithFlags(&ix->fill_streams[i], cudaStreamNonBlocking) != cudaSuccess) return bail(GORIO_ERR_CUDA);
+  for (int i = 0; i < kFillEvents; ++i)
+    if (cudaEventCreateWithFlags(&ix->fill_events[i], cudaEventDisableTiming) != cudaSuccess) return bail(GORIO_ERR_CUDA);
   ix->proxy = std::thread(proxy_main, ix);
   *out = ix;
   return GORIO_OK;
@@ -591,6 +646,8 @@ int gorio_index_close(gorio_index *ix) {
   if (ix->hctl_h) cudaFreeHost(ix->hctl_h);
   if (ix->own_stream) cudaStreamDestroy(ix->own_stream);
   if (ix->done_ev) cudaEventDestroy(ix->done_ev);
+  for (int i = 0; i < kFillStreams; ++i) if (ix->fill_streams[i]) cudaStreamDestroy(ix->fill_streams[i]);
+  for (int i = 0; i < kFillEvents; ++i) if (ix->fill_events[i]) cudaEventDestroy(ix->fill_events[i]);
   if (ix->registered_pages) cudaHostUnregister((void *)ix->desc.host_pages);
   delete ix;
   return GORIO_OK;
@@ -602,6 +659,7 @@ int gorio_cache_config(gorio_index *ix, const gorio_cache_cfg *cfg) {
   if (cfg->capacity_pages < 16 || cfg->max_outstanding < 1)
     return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: capacity >= 16, max_outstanding >= 1");
   if (cfg->granularity > GORIO_GRAN_RECORD) return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: unknown granularity");
+  if (cfg->copy_mode > GORIO_COPY_ENGINE) return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: unknown copy_mode");
   if (cfg->granularity == GORIO_GRAN_RECORD && cfg->preload)
     return fail(ix, GORIO_ERR_INVALID_ARG, "cache_config: preload needs page granularity");
   u64 cap = cfg->capacity_pages < ix->n_pages ? cfg->capacity_pages : ix->n_pages;
@@ -636,6 +694,10 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   if (!queries_dev || !out_ids_dev || !out_dists_dev || nq < 1 || K < 1 || K > L || L > 256 || W < 1 ||
       W > 16 || (u64)W * ix->desc.max_degree > 1024)
     return fail(ix, GORIO_ERR_INVALID_ARG, "search: need 1 <= K <= L <= 256, 1 <= W <= 16, W*max_degree <= 1024");
+  // the kernels read and write 32-bit words through these pointers: a misaligned one would trap
+  if ((((uintptr_t)queries_dev | (uintptr_t)out_ids_dev | (uintptr_t)out_dists_dev | (uintptr_t)out_pages_distinct_dev |
+        (uintptr_t)out_counters_dev) & 3u) != 0)
+    return fail(ix, GORIO_ERR_INVALID_ARG, "search: queries and outputs must be at least 4-byte aligned");
   if (!ix->cache_ready) return fail(ix, GORIO_ERR_STATE, "search: call gorio_cache_config first");
   CK(cudaSetDevice(ix->dev));
   cudaStream_t stream = (cudaStream_t)cuda_stream;
@@ -686,6 +748,10 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   CK(cudaStreamSynchronize(stream));
   ix->host_search_ns += (u64)std::chrono::duration_cast<std::chrono::nanoseconds>(Clock::now() - t_begin).count();
   print_diagnostics(c, h);
+  if (ix->px_error.load() == 2) {
+    for (int i = 0; i < kFillStreams; ++i) cudaStreamSynchronize(ix->fill_streams[i]);
+    return fail(ix, GORIO_ERR_CUDA, "proxy: a page copy or its completion event failed");
+  }
   if (ix->px_error.load()) return fail(ix, GORIO_ERR_INTERNAL, "proxy: descriptor out of range");
   if (h.status != 0 || h.stop != 1) return device_failure(ix, h, nq);
   ix->cache_dirty = false;

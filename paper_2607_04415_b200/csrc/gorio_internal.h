@@ -141,6 +141,8 @@ struct Ctx {
   u32 vec128;      // 1: vectors are whole 16-byte chunks (<= 24) and query rows are 16-byte aligned
   u32 blocking;    // 1: a warp waits in place for its query's pages instead of yielding
   u32 prof;        // debug: 1 = account warp time per query phase step in stats[S_P_*]
+  u32 dma_fill;    // 1: the proxy fills slots with the copy engine and publishes a completion only after
+                   //    the copy has landed: no warp copies pages and `filled` is not used
   u32 identity;    // 1: every unit is resident in the slot of the same number and nothing can be
                    //    evicted (whole index preloaded): lookups and hit validation are skipped
 };

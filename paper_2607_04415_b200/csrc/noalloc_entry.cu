@@ -73,8 +73,12 @@ extern "C" int gorio_search_resident_noalloc(const gorio_index_desc *d, const vo
   const u64 nb = (u64)d->dim * esz + 4 + 4ull * d->max_degree;
   if (d->dtype > GORIO_DTYPE_F32 || d->page_bytes != kPageBytes || d->dim == 0 || d->dim % 4 != 0 ||
       d->max_degree == 0 || d->nodes_per_page == 0 || nb * d->nodes_per_page > kPageBytes || d->n_nodes == 0 ||
-      d->entry_id >= d->n_nodes)
+      d->n_nodes >= (1ull << 31) || d->entry_id >= d->n_nodes)
     return na_fail(GORIO_ERR_INVALID_ARG, "noalloc search: bad index description");
+  // the kernels read and write 32-bit words through these pointers: a misaligned one would trap
+  if ((((uintptr_t)pages_dev | (uintptr_t)queries_dev | (uintptr_t)out_ids_dev | (uintptr_t)out_dists_dev |
+        (uintptr_t)out_pages_distinct_dev) & 3u) != 0)
+    return na_fail(GORIO_ERR_INVALID_ARG, "noalloc search: pages, queries and outputs must be at least 4-byte aligned");
   if (d->pq_m != 0) return na_fail(GORIO_ERR_INVALID_ARG, "noalloc search: PQ navigation is not supported here");
   const u64 n_pages = (d->n_nodes + d->nodes_per_page - 1) / d->nodes_per_page;
   if (n_pages > kNaMaxPages)

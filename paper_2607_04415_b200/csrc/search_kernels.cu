@@ -2,8 +2,8 @@
 //
 // One persistent kernel runs every query of a batch.  Warps are the execution slots: a
 // warp pops a runnable query slot from a queue in HBM, advances it by one or more phases,
-// and parks it when it has to wait for pages (paper Section 3.3: blocks "claim work,
-// execute graph traversal, and either finish a query or mark it pending on a missing page").
+// and parks it when it has to wait for pages (paper Section 3.3: a search block takes a
+// query, runs its traversal, and ends by either completing it or leaving it pending on a page).
 //
 // Data flow of one query iteration:
 //   PH_EVAL  complete -> merge the scored candidates into the sorted L-entry list, pick the

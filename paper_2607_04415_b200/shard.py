@@ -24,3 +24,28 @@ def gather_results(local: torch.Tensor, nq: int):
     parts = [torch.empty_like(buf) for _ in range(world)]
     dist.all_gather(parts, buf)
     return torch.cat([p[:s] for p, s in zip(parts, sizes)], 0)
+
+
+def free_port() -> int:
+    """A TCP port that is free on 127.0.0.1 right now (for the rendezvous of a local launch)."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(n_ranks: int, script: str, argv, env=None, timeout=None) -> int:
+    """Run `script argv...` as n_ranks processes of one node, one per GPU, the way a launcher
+    would: `python -m torch.distributed.run --nnodes=1 --nproc-per-node n --master-addr 127.0.0.1
+    --master-port <free port> script argv...`, so that every child finds RANK, LOCAL_RANK,
+    WORLD_SIZE and MASTER_* in its environment.  Returns the launcher's exit code (non-zero if
+    any rank failed).  The children share nothing on the device: no collective is on the data path."""
+    import os
+    import subprocess
+    import sys
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={int(n_ranks)}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), script] + list(argv)
+    e = dict(os.environ if env is None else env)
+    for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE"):      # the launcher sets these for its children
+        e.pop(k, None)
+    return subprocess.run(cmd, env=e, timeout=timeout).returncode

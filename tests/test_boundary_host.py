@@ -111,6 +111,96 @@ def test_two_rank_gloo_gather_restores_global_order():
     assert tmax == 2.0
 
 
+def test_binding_rejects_wrong_shapes_types_and_sizes_before_any_pointer_is_passed():
+    """The library sees raw pointers only, so the binding checks what it cannot: a wrong-shaped,
+    wrong-typed, non-contiguous, misplaced or misaligned tensor is an INVALID_ARG error, never
+    an out-of-bounds device access."""
+    import paper_2607_04415_b200.binding as b
+    good = torch.zeros((8, 128), dtype=torch.uint8)
+    for bad in (torch.zeros(128, dtype=torch.uint8),                  # not 2-D
+                torch.zeros((8, 64), dtype=torch.uint8),              # wrong width
+                torch.zeros((8, 128), dtype=torch.float32),           # wrong element type
+                torch.zeros((128, 8), dtype=torch.uint8).t(),         # right shape, not contiguous
+                good):                                                # not on a CUDA device
+        with pytest.raises(b.GorioError) as e:
+            b.check_queries(bad, 128, "u8", 0)
+        assert e.value.status == 1
+    with pytest.raises(b.GorioError) as e:
+        b.check_queries(torch.zeros((8, 96), dtype=torch.uint8), 96, "f32")
+    assert e.value.status == 1
+    cpu = torch.device("cpu")
+    pages = torch.zeros(4 * 4096, dtype=torch.uint8)
+    for args in ((pages, 0, 1), (pages, 4, 0), (pages.to(torch.int32), 4, 1), (pages[::2], 2, 1)):
+        with pytest.raises(b.GorioError) as e:
+            b.check_resident_pages(args[0], args[1], args[2], cpu)
+        assert e.value.status == 1
+
+
+def test_c_entries_reject_misaligned_pointers_and_oversized_indexes_without_a_gpu(lib):
+    import paper_2607_04415_b200.binding as b
+    d = b._IndexDesc()
+    d.n_nodes, d.dim, d.dtype, d.max_degree, d.nodes_per_page, d.page_bytes, d.entry_id = 100, 128, 0, 32, 1, 4096, 0
+    fake = 0x10000                                        # never dereferenced: validation fails first
+    call = lambda desc, pages, q, ids: lib.gorio_search_resident_noalloc(ctypes.byref(desc), pages, q, 4, 10, 64, 4,
+                                                                         ids, fake, None, None)
+    assert call(d, fake + 2, fake, fake) == 1             # pages not 4-byte aligned
+    assert call(d, fake, fake + 1, fake) == 1             # queries not 4-byte aligned
+    assert call(d, fake, fake, fake + 2) == 1             # outputs not 4-byte aligned
+    assert b"aligned" in lib.gorio_last_error(None)
+    d.n_nodes = 1 << 31                                   # the list key keeps ids in 31 bits
+    assert call(d, fake, fake, fake) == 1
+    d.n_nodes = (1 << 64) - 1                             # n_nodes + nodes_per_page - 1 must not wrap
+    assert call(d, fake, fake, fake) == 1
+
+
+def _stub_rank_script(tmp_path):
+    p = tmp_path / "stub_rank.py"
+    p.write_text(
+        "import os, sys, torch, torch.distributed as dist\n"
+        "dist.init_process_group('gloo')\n"
+        "r, w = dist.get_rank(), dist.get_world_size()\n"
+        "assert r == int(os.environ['RANK']) and w == int(os.environ['WORLD_SIZE']) == int(sys.argv[1])\n"
+        "assert int(os.environ['LOCAL_RANK']) == r and os.environ['MASTER_ADDR'] == '127.0.0.1'\n"
+        "t = torch.tensor([float(r + 1)]); dist.all_reduce(t, op=dist.ReduceOp.MAX)\n"
+        "open(os.path.join(sys.argv[2], f'rank{r}.txt'), 'w').write(f'{w} {t.item()}')\n"
+        "dist.destroy_process_group()\n"
+        "sys.exit(3 if (len(sys.argv) > 3 and r == 1) else 0)\n")
+    return str(p)
+
+
+def test_spawn_ranks_starts_one_process_per_rank_with_the_launcher_environment(tmp_path):
+    from paper_2607_04415_b200.shard import spawn_ranks
+    script = _stub_rank_script(tmp_path)
+    assert spawn_ranks(2, script, ["2", str(tmp_path)], timeout=300) == 0
+    for r in range(2):
+        assert (tmp_path / f"rank{r}.txt").read_text() == "2 2.0"
+    # a failing rank makes the launch fail
+    assert spawn_ranks(2, script, ["2", str(tmp_path), "fail"], timeout=300) != 0
+
+
+def test_bench_reference_arm_with_two_gpus_still_prints_one_line():
+    import json
+    import subprocess
+    import sys
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--config", "3",
+                          "--scale", "0.01", "--nq", "64", "--steps", "1", "--warmup", "1"],
+                         capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-800:]
+    lines = [ln for ln in out.stdout.strip().splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
+
+
+def test_bench_refuses_a_world_size_that_differs_from_gpus():
+    import subprocess
+    import sys
+    env = dict(os.environ, RANK="0", LOCAL_RANK="0", WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT="1")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--steps", "1"],
+                         capture_output=True, text=True, timeout=300, cwd=ROOT, env=env)
+    assert out.returncode != 0 and "--gpus 4" in (out.stderr + out.stdout)
+
+
 def test_bench_reference_arm_prints_the_contract_line_on_cpu():
     """`bench.py --impl reference` times the oracle and needs no GPU: one JSON line with the
     contract's keys, on a shrunken workload so that the CPU suite stays short."""

@@ -9,7 +9,8 @@ from oracle import OracleIndex
 from workloads import make_config, make_workload, train_pq, write_page_store
 from workloads import node_bytes as nbytes
 
-from test_gpu_parity import _assert_exact, _check_stats_invariants, _fp32_parity, _gpu_search, _u32, gorio  # noqa: F401
+from helpers import fp32_parity as _fp32_parity
+from test_gpu_parity import _assert_exact, _check_stats_invariants, _gpu_search, _u32, gorio  # noqa: F401
 
 pytestmark = pytest.mark.gpu
 

@@ -20,4 +20,5 @@ from .synthetic import (  # noqa: F401
     make_workload,
     make_config,
     recall_at_k,
+    workload_key,
 )

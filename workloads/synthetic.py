@@ -395,6 +395,11 @@ class Workload:
         return int(np.floor(self.cache_frac * self.n_pages))
 
 
+def workload_key(cfg: int, N: int, npp: int, nq: int, L: int, W: int, slots: int) -> str:
+    """Name of a (workload, search parameters, cache size) combination in stored result files."""
+    return f"cfg{cfg}:N={N}:npp={npp}:nq={nq}:L={L}:W={W}:slots={slots}"
+
+
 def make_workload(name, kind, N, C, nq, d, k, n_rand, npp, clustered_knn, cross_only,
                   with_pq=False, with_gt=True, device=None, seed_q=1, **search):
     """Generate vectors, graph, page store (and optionally PQ and ground truth)."""
