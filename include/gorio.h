@@ -148,6 +148,11 @@ enum { GORIO_GRAN_PAGE = 0, GORIO_GRAN_RECORD = 1 };
  *   request_backlog  most requests posted to the proxy and not yet arrived; 0 = default
  *                    min(4 * max_outstanding, 1024), never below max_outstanding.  More than the proxy can have in service only queues
  *                    in the ring while occupying cache slots that could hold resident pages.
+ *   no_fast_path     1 = do not use the whole-index-resident fast path.  When the whole index was
+ *                    preloaded (nothing can miss) a warp normally runs each query from admission
+ *                    to output without parking it, with the list in registers and the candidates
+ *                    in shared memory; with this flag such a search goes through the general
+ *                    park-and-resume machinery instead.  Results are identical; for comparisons.
  *   blocking         1 = ablation: a warp that misses keeps its query and waits in place for
  *                    the pages (the demand-paging baseline of Section 5.1) instead of parking
  *                    the query and taking another; results are identical, only slower.
@@ -160,7 +165,7 @@ typedef struct {
   uint32_t stash_entries;
   uint32_t blocking;
   uint32_t request_backlog;
-  uint32_t reserved;
+  uint32_t no_fast_path;
 } gorio_tuning;
 
 /*

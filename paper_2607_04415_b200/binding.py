@@ -46,7 +46,7 @@ class _Tuning(ctypes.Structure):
     _fields_ = [("max_inflight", ctypes.c_uint32), ("visited_capacity", ctypes.c_uint32),
                 ("warps_per_block", ctypes.c_uint32), ("blocks_per_sm", ctypes.c_uint32),
                 ("stash_entries", ctypes.c_uint32), ("blocking", ctypes.c_uint32),
-                ("request_backlog", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+                ("request_backlog", ctypes.c_uint32), ("no_fast_path", ctypes.c_uint32)]
 
 
 _STAT_FIELDS = ["pages_hit", "pages_missed", "pages_fetched", "dedupe_joins", "evictions", "retries",
@@ -198,9 +198,9 @@ class Index:
         self._check(self._lib.gorio_cache_config(self._h, ctypes.byref(cfg)))
 
     def set_tuning(self, max_inflight=0, visited_capacity=0, warps_per_block=0, blocks_per_sm=0, stash_entries=0,
-                   blocking=0, request_backlog=0):
+                   blocking=0, request_backlog=0, no_fast_path=0):
         t = _Tuning(max_inflight, visited_capacity, warps_per_block, blocks_per_sm, stash_entries, int(blocking),
-                    request_backlog, 0)
+                    request_backlog, int(no_fast_path))
         self._check(self._lib.gorio_set_tuning(self._h, ctypes.byref(t)))
 
     def search(self, queries: torch.Tensor, K: int, L: int, W: int, want_counters=True, stream=None):

@@ -60,6 +60,8 @@ __device__ bool recycle_slot(const Ctx &c, u32 qs, u32 lane) {
 }
 
 __device__ void copy_page(const Ctx &c, u32 idx, u32 lane);
+template <bool PQ> __device__ void resident_worker(const Ctx &c, u32 lane, u32 *lut, u32 *ws);
+__host__ __device__ inline u32 resident_warp_words(u32 WR);
 __device__ bool warp_ticket(int *count, u32 *head, u32 &idx, u32 lane);
 
 // One unit of the work that keeps pages moving, in priority order: execute a copy the proxy
@@ -331,6 +333,12 @@ __global__ void __launch_bounds__(MAXT, 1) search_kernel(const Ctx c) {
   const u32 lane = lane_id(), warp = threadIdx.x >> 5;
   if (blockIdx.x == 0 && warp == 0) { poller(c, lane); return; }
   u32 *lut = PQ ? smem_lut + (u64)warp * c.pq_m * kPqLutWords : nullptr;
+  if (c.resident_fast) {                   // whole index resident: queries run start to end on one warp
+    const u32 n_warps = blockDim.x >> 5;
+    u32 *ws = smem_lut + (PQ ? (u64)n_warps * c.pq_m * kPqLutWords : 0) + (u64)warp * resident_warp_words(c.WR);
+    resident_worker<PQ>(c, lane, lut, ws);
+    return;
+  }
   const u64 t0 = globaltimer();
   u32 idle = 0;
   // where the worker warps' time goes (ns, summed over warps): arrivals, query phases, idle

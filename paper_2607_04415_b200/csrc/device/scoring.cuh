@@ -92,90 +92,65 @@ __device__ __forceinline__ void complete_items(const Ctx &c, u32 qs, u32 n) {
   else if (old < n) raise(c, 8, 0x61, qs, old, n);
 }
 
-// Score the nodes of `eval_mask` (lane i holds node i's query id, node id and cache slot) with
-// 128-bit loads: the warp works as four 8-lane groups, each group scores one node per round,
-// lane t of a group handling the 16-byte chunks t, t+8, t+16 of the vector.  Records are only
-// 4-byte aligned inside a page (388- or 644-byte nodes), so a chunk is assembled from the two
-// 16-byte-aligned pieces that cover it by word selection; query rows are 16-byte aligned.
-// ROUNDS nodes per group are loaded before any is reduced.  Returns the distance (u32 bits) to
-// the lanes of eval_mask.
-__device__ __forceinline__ u32 pick_word(const uint4 &a, const uint4 &b, u32 i) {
-  // word i (0..6) of the 8-word sequence a.x a.y a.z a.w b.x b.y b.z b.w
-  const u32 lo = (i & 2u) ? ((i & 1u) ? a.w : a.z) : ((i & 1u) ? a.y : a.x);
-  const u32 hi = (i & 2u) ? ((i & 1u) ? b.w : b.z) : ((i & 1u) ? b.y : b.x);
-  return (i & 4u) ? hi : lo;
-}
-
-template <int CH, int ROUNDS>
-__device__ __forceinline__ u32 score_group128(const Ctx &c, u32 eval_mask, u32 qid, u32 node, u32 slot, u32 lane) {
-  const u32 grp = lane >> 3, t = lane & 7u;
-  const u32 nchunk = c.vec_bytes >> 4;
-  u32 dist = 0;
-  for (u32 m = eval_mask; m;) {
-    uint4 A[ROUNDS][CH], B[ROUNDS][CH], Q[ROUNDS][CH];
-    u32 src[ROUNDS], sw[ROUNDS];
-    bool valid[ROUNDS];
+// Lane-per-node scoring with 128-bit loads: every active lane scores its OWN node against its own
+// query, so up to 32 nodes are in flight per pass and no lane waits on another's data.  A vector
+// is handled in blocks of eight 16-byte chunks: the lane loads the nine aligned chunks that cover
+// the block (records are only 4-byte aligned in a page), shifts them down by its own misalignment
+// (0..3 words, two conditional-move levels, no dynamic register indexing) and reduces against the
+// query's chunks, which are 16-byte aligned.  uint8: |a-b| per byte and a 4-way dot product into
+// one exact u32.  fp32: eight accumulators, accumulator t taking the chunks t, t+8, t+16 in that
+// order, combined as ((a0+a4)+(a2+a6))+((a1+a5)+(a3+a7)) -- the summation order of an 8-lane
+// butterfly, so the value does not depend on which path scored the node.
+__device__ __forceinline__ u32 lane_score128(const Ctx &c, bool active, u32 qid, u32 node, u32 slot) {
+  const u32 nchunk = c.vec_bytes >> 4;                       // <= 24 (checked on the host: vec128)
+  const u32 off = rec_off(c, node);
+  const u32 sw = (off & 15u) >> 2;
+  const uint4 *base = (const uint4 *)(c.slot_data + (u64)slot * c.slot_bytes + (off & ~15u));
+  const uint4 *q4 = (const uint4 *)((const u8 *)c.queries + (u64)qid * c.vec_bytes);
+  const u32 ncha = nchunk + (sw ? 1u : 0u);                  // aligned chunks that hold the vector
+  const bool s2 = (sw & 2u) != 0u, s1 = (sw & 1u) != 0u;
+  u32 acc_u = 0;
+  float acc_f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  uint4 carry = make_uint4(0, 0, 0, 0);
+  for (u32 b0 = 0; b0 < nchunk; b0 += 8) {
+    u32 w[36];
+    {
+      uint4 A[9];
+      A[0] = carry;
 #pragma unroll
-    for (int r = 0; r < ROUNDS; ++r) {
-      const u32 sel = __fns(m, 0, (int)(r * 4 + grp) + 1);      // this group's node of this round
-      valid[r] = sel < 32u;
-      src[r] = valid[r] ? sel : 0u;
-      const u32 s_qid = __shfl_sync(0xffffffffu, qid, src[r]), s_node = __shfl_sync(0xffffffffu, node, src[r]);
-      const u32 s_slot = __shfl_sync(0xffffffffu, slot, src[r]);
-      const u32 off = rec_off(c, s_node);
-      sw[r] = (off & 15u) >> 2;
-      const u8 *base = c.slot_data + (u64)s_slot * c.slot_bytes + (off & ~15u);
-      const u8 *q = (const u8 *)c.queries + (u64)s_qid * c.vec_bytes;
-#pragma unroll
-      for (int k = 0; k < CH; ++k) {
-        const u32 ch = t + 8u * (u32)k;
-        const bool in = valid[r] && ch < nchunk;
-        A[r][k] = in ? __ldcg((const uint4 *)(base + 16u * ch)) : make_uint4(0, 0, 0, 0);
-        B[r][k] = (in && sw[r]) ? __ldcg((const uint4 *)(base + 16u * ch + 16u)) : make_uint4(0, 0, 0, 0);
-        Q[r][k] = in ? __ldg((const uint4 *)(q + 16u * ch)) : make_uint4(0, 0, 0, 0);
+      for (int k = 0; k < 9; ++k) {
+        if (k == 0 && b0 != 0) continue;                     // carried over from the previous block
+        const u32 a = b0 + (u32)k;
+        A[k] = (active && a < ncha) ? __ldcg(base + a) : make_uint4(0, 0, 0, 0);
       }
+      carry = A[8];
+#pragma unroll
+      for (int k = 0; k < 9; ++k) { w[4 * k] = A[k].x; w[4 * k + 1] = A[k].y; w[4 * k + 2] = A[k].z; w[4 * k + 3] = A[k].w; }
     }
 #pragma unroll
-    for (int r = 0; r < ROUNDS; ++r) {
-      u32 d;
-      if (c.dtype == 0) {
-        u32 acc = 0;
+    for (int i = 0; i < 34; ++i) w[i] = s2 ? w[i + 2] : w[i];
 #pragma unroll
-        for (int k = 0; k < CH; ++k) {
-          const u32 qq[4] = {Q[r][k].x, Q[r][k].y, Q[r][k].z, Q[r][k].w};
+    for (int i = 0; i < 32; ++i) w[i] = s1 ? w[i + 1] : w[i];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) { const u32 x = __vabsdiffu4(pick_word(A[r][k], B[r][k], sw[r] + i), qq[i]); acc = __dp4a(x, x, acc); }
-        }
+    for (int t = 0; t < 8; ++t) {
+      if (b0 + (u32)t < nchunk) {                            // warp-uniform
+        const uint4 qv = active ? __ldg(q4 + b0 + t) : make_uint4(0, 0, 0, 0);
+        const u32 qq[4] = {qv.x, qv.y, qv.z, qv.w};
+        if (c.dtype == 0) {
 #pragma unroll
-        for (int o = 4; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        d = acc;
-      } else {
-        float acc = 0.f;
-#pragma unroll
-        for (int k = 0; k < CH; ++k) {
-          const u32 qq[4] = {Q[r][k].x, Q[r][k].y, Q[r][k].z, Q[r][k].w};
+          for (int i = 0; i < 4; ++i) { const u32 x = __vabsdiffu4(w[4 * t + i], qq[i]); acc_u = __dp4a(x, x, acc_u); }
+        } else {
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const float x = __uint_as_float(qq[i]) - __uint_as_float(pick_word(A[r][k], B[r][k], sw[r] + i));
-            acc = fmaf(x, x, acc);
+            const float x = __uint_as_float(qq[i]) - __uint_as_float(w[4 * t + i]);
+            acc_f[t] = fmaf(x, x, acc_f[t]);
           }
         }
-#pragma unroll
-        for (int o = 4; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        d = __float_as_uint(acc);
-      }
-      // hand each group's result to the lane that owns the node
-#pragma unroll
-      for (int g = 0; g < 4; ++g) {
-        const u32 dg = __shfl_sync(0xffffffffu, d, g * 8);
-        const u32 owner = __shfl_sync(0xffffffffu, valid[r] ? src[r] : 0xFFu, g * 8);
-        if (lane == owner) dist = dg;
       }
     }
-#pragma unroll
-    for (int i = 0; i < 4 * ROUNDS; ++i) m &= m - 1;      // the nodes just scored
   }
-  return dist;
+  if (c.dtype == 0) return acc_u;
+  return __float_as_uint(((acc_f[0] + acc_f[4]) + (acc_f[2] + acc_f[6])) + ((acc_f[1] + acc_f[5]) + (acc_f[3] + acc_f[7])));
 }
 
 // Consume up to 32 items at once: lane i holds item i = (query slot, item index, cache slot) if
@@ -195,10 +170,7 @@ __device__ __noinline__ void consume_group(const Ctx &c, u32 mask, u32 qs, u32 j
   const u32 words = c.vec_bytes >> 2;
   const u32 eval_mask = words <= 96u ? __ballot_sync(0xffffffffu, mine && phase == PH_EVAL) : 0u;
   u32 dist = 0;
-  if (c.vec128 && eval_mask) {
-    if (c.vec_bytes <= 128u) dist = score_group128<1, 2>(c, eval_mask, qid, node, slot, lane);
-    else dist = score_group128<3, 1>(c, eval_mask, qid, node, slot, lane);
-  }
+  if (c.vec128 && eval_mask) dist = lane_score128(c, (eval_mask >> lane) & 1u, qid, node, slot);
   for (u32 m = c.vec128 ? 0u : eval_mask; m;) {
     u32 src[4], a[4][3], b[4][3];
     int ng = 0;

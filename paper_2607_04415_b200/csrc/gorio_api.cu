@@ -375,9 +375,12 @@ int setup_cache(gorio_index *ix) {
   return GORIO_OK;
 }
 
-int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W) {
+// slot_cap: most query slots this search can use at once (the worker warps of the resident fast
+// path, which run one query each; otherwise no limit beyond max_inflight)
+int ensure_qstate(gorio_index *ix, u32 nq, u32 K, u32 L, u32 W, u32 slot_cap) {
   const u32 R = ix->desc.max_degree, WR = W * R;
-  const u32 max_inflight = ix->tune.max_inflight ? ix->tune.max_inflight : 16384u;
+  u32 max_inflight = ix->tune.max_inflight ? ix->tune.max_inflight : 16384u;
+  if (slot_cap && slot_cap < max_inflight) max_inflight = slot_cap;
   const u32 slots = nq < max_inflight ? nq : max_inflight;
   // exact visited set per query: a bitmap over the nodes when that is no larger than the hash set
   // (one atomicOr, no probing, never full), else the hash set (config 5: 10M nodes)
@@ -442,6 +445,15 @@ thread_local char g_global_error[256] = "";
 const char *kDeviceErr[] = {"", "", "", "", "", "device wait expired", "per-query capacity exhausted",
                             "corrupt index page", "internal state-machine check failed"};
 
+// whole index preloaded page by page: slot p holds page p and no request can ever be posted
+bool whole_index_resident(const gorio_index *ix) {
+  return !ix->record_mode && ix->preloaded == ix->n_units && ix->n_slots == ix->n_units;
+}
+// ... and the search fits the fast path's fixed shapes (PQ: the rerank pool is one key per lane)
+bool resident_fast_path(const gorio_index *ix, u32 K, u32 W) {
+  return whole_index_resident(ix) && !ix->tune.no_fast_path && W <= 16u && (ix->desc.pq_m == 0 || K + W <= 32u);
+}
+
 // Everything the kernels need for this search, gathered into the by-value context.
 void fill_ctx(gorio_index *ix, const void *queries_dev, u32 nq, u32 K, u32 L, u32 W, u32 *out_ids_dev, void *out_dists_dev,
               u32 *out_pages_distinct_dev, u32 *out_counters_dev) {
@@ -478,14 +490,18 @@ void fill_ctx(gorio_index *ix, const void *queries_dev, u32 nq, u32 K, u32 L, u3
   c.prof = std::getenv("GORIO_PROFILE") ? 1u : 0u;
   // whole index preloaded page by page: slot p holds page p and no request can ever be posted
   c.dma_fill = ix->cfg.copy_mode == GORIO_COPY_ENGINE ? 1u : 0u;
-  c.identity = (!ix->record_mode && ix->preloaded == ix->n_units && ix->n_slots == ix->n_units) ? 1u : 0u;
+  c.identity = whole_index_resident(ix) ? 1u : 0u;
+  c.resident_fast = resident_fast_path(ix, K, W) ? 1u : 0u;
 }
 
-// Launch geometry of the persistent kernel: blocks and warps per block.
-int launch_geometry(gorio_index *ix, u32 nq, u32 *blocks_out, u32 *warps_out) {
+// Launch geometry of the persistent kernel: blocks and warps per block.  Needs only the index, the
+// cache and (K, W); runs before the query state is sized.
+int launch_geometry(gorio_index *ix, u32 nq, u32 K, u32 W, u32 *blocks_out, u32 *warps_out) {
   const gorio_index_desc &d = ix->desc;
   // launch geometry: one block per SM by default
   const bool pq = d.pq_m != 0;
+  Ctx g{};                        // the fields the shared-memory size depends on
+  g.pq_m = d.pq_m; g.WR = W * d.max_degree; g.resident_fast = resident_fast_path(ix, K, W) ? 1u : 0u;
   // default warps per SM: 16 when pages will be missed (more warps lengthen every copy and arrival);
   // with every page resident one warp carries one query at a time, so no more than there are
   // queries per SM (fewer idle warps polling the queues), within 8..24
@@ -493,16 +509,18 @@ int launch_geometry(gorio_index *ix, u32 nq, u32 *blocks_out, u32 *warps_out) {
   if (ix->n_slots >= ix->n_units) {
     auto_warps = (nq + (u32)ix->n_sms - 1) / (u32)ix->n_sms;
     auto_warps = auto_warps < 8u ? 8u : (auto_warps > 24u ? 24u : auto_warps);
+    if (g.resident_fast && auto_warps > 16u) auto_warps = 16u;     // the fast path wants the 128-register build
   }
-  u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 10u : auto_warps);
-  if (pq) {      // one table per warp in shared memory; the PQ kernel is built for at most 12 warps
-    u32 lim = (220u * 1024u) / (d.pq_m * kPqLutWords * 4u);
-    if (lim > 12u) lim = 12u;
+  u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? (g.resident_fast ? 12u : 10u) : auto_warps);
+  const size_t per_warp = search_smem_per_warp(g);
+  if (per_warp) {                 // per-warp tables / candidate areas in shared memory
+    u32 lim = (u32)((220u * 1024u) / per_warp);
+    if (pq && lim > 12u) lim = 12u;      // the PQ kernel is built for at most 12 warps
     if (warps > lim) warps = lim;
   }
   if (warps < 2) return fail(ix, GORIO_ERR_INVALID_ARG, "search: need at least 2 warps per block (the poller and a worker)");
   int occ = 0;
-  CK(search_occupancy(d.pq_m, warps, &occ));
+  CK(search_occupancy(g, warps, &occ));
   if (occ < 1) return fail(ix, GORIO_ERR_INVALID_ARG, "search: launch geometry does not fit an SM");
   u32 bps = ix->tune.blocks_per_sm ? ix->tune.blocks_per_sm : 1u;
   if ((int)bps > occ) bps = (u32)occ;
@@ -706,14 +724,16 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
     int st = setup_cache(ix);
     if (st != GORIO_OK) return st;
   }
-  int st = ensure_qstate(ix, nq, K, L, W);
+  u32 blocks = 0, warps = 0;
+  int st = launch_geometry(ix, nq, K, W, &blocks, &warps);
+  if (st != GORIO_OK) return st;
+  // on the resident fast path a warp carries one query from start to end, so no more query slots
+  // than worker warps are ever in use (less state to clear per call)
+  st = ensure_qstate(ix, nq, K, L, W, resident_fast_path(ix, K, W) ? blocks * warps : 0u);
   if (st != GORIO_OK) return st;
 
   fill_ctx(ix, queries_dev, nq, K, L, W, out_ids_dev, out_dists_dev, out_pages_distinct_dev, out_counters_dev);
   Ctx &c = ix->ctx;
-  u32 blocks = 0, warps = 0;
-  st = launch_geometry(ix, nq, &blocks, &warps);
-  if (st != GORIO_OK) return st;
 
   // reset the host-visible rings while the proxy is idle
   std::memset(ix->ring_h, 0, (size_t)ix->ring_cap * 8);

@@ -143,6 +143,8 @@ struct Ctx {
   u32 prof;        // debug: 1 = account warp time per query phase step in stats[S_P_*]
   u32 dma_fill;    // 1: the proxy fills slots with the copy engine and publishes a completion only after
                    //    the copy has landed: no warp copies pages and `filled` is not used
+  u32 resident_fast; // 1 (needs identity): a warp runs each query from admission to output without parking it;
+                   //    list in registers, candidates in shared memory (device/resident.cuh)
   u32 identity;    // 1: every unit is resident in the slot of the same number and nothing can be
                    //    evicted (whole index preloaded): lookups and hit validation are skipped
 };
@@ -151,7 +153,8 @@ struct Ctx {
 cudaError_t preload_kernels();
 cudaError_t launch_init(const Ctx &c, cudaStream_t s);
 cudaError_t launch_search(const Ctx &c, u32 blocks, u32 warps_per_block, cudaStream_t s);
-cudaError_t search_occupancy(u32 pq_m, u32 warps_per_block, int *blocks_per_sm);
+cudaError_t search_occupancy(const Ctx &c, u32 warps_per_block, int *blocks_per_sm);
+size_t search_smem_per_warp(const Ctx &c);
 cudaError_t launch_cache_reset(const Ctx &c, u32 preloaded_pages, cudaStream_t s);
 
 }  // namespace gorio

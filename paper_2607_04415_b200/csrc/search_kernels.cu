@@ -28,6 +28,7 @@
 #include "device/list.cuh"
 #include "device/pq.cuh"
 #include "device/scheduler.cuh"
+#include "device/resident.cuh"
 
 namespace gorio {
 
@@ -93,30 +94,38 @@ cudaError_t launch_cache_reset(const Ctx &c, u32 preloaded, cudaStream_t s) {
   return cudaGetLastError();
 }
 
-static size_t search_smem(const Ctx &c, u32 warps) { return c.pq_m ? (size_t)warps * c.pq_m * kPqLutWords * 4 : 0; }
+// Dynamic shared memory per warp: the PQ distance table, and on the resident fast path the
+// warp's candidate area.
+size_t search_smem_per_warp(const Ctx &c) {
+  return (c.pq_m ? (size_t)c.pq_m * kPqLutWords * 4 : 0) + (c.resident_fast ? (size_t)resident_warp_words(c.WR) * 4 : 0);
+}
 
-cudaError_t search_occupancy(u32 pq_m, u32 warps_per_block, int *blocks_per_sm) {
-  if (pq_m) {
-    const size_t smem = (size_t)warps_per_block * pq_m * kPqLutWords * 4;
-    cudaError_t e = cudaFuncSetAttribute(search_kernel<true, 384>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<true, 384>, warps_per_block * 32, smem);
-  }
-  if (warps_per_block <= 16)
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<false, 512>, warps_per_block * 32, 0);
-  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<false, 768>, warps_per_block * 32, 0);
+template <typename K>
+static cudaError_t occupancy_of(K kernel, u32 threads, size_t smem, int *blocks_per_sm) {
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, kernel, threads, smem);
+}
+
+cudaError_t search_occupancy(const Ctx &c, u32 warps_per_block, int *blocks_per_sm) {
+  const size_t smem = search_smem_per_warp(c) * warps_per_block;
+  if (c.pq_m) return occupancy_of(search_kernel<true, 384>, warps_per_block * 32, smem, blocks_per_sm);
+  if (warps_per_block <= 16) return occupancy_of(search_kernel<false, 512>, warps_per_block * 32, smem, blocks_per_sm);
+  return occupancy_of(search_kernel<false, 768>, warps_per_block * 32, smem, blocks_per_sm);
 }
 
 cudaError_t launch_search(const Ctx &c, u32 blocks, u32 warps_per_block, cudaStream_t s) {
-  const size_t smem = search_smem(c, warps_per_block);
+  const size_t smem = search_smem_per_warp(c) * warps_per_block;
+  cudaError_t e;
   if (c.pq_m) {
-    cudaError_t e = cudaFuncSetAttribute(search_kernel<true, 384>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(search_kernel<true, 384>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
     search_kernel<true, 384><<<blocks, warps_per_block * 32, smem, s>>>(c);
   } else if (warps_per_block <= 16) {
-    search_kernel<false, 512><<<blocks, warps_per_block * 32, 0, s>>>(c);
+    if ((e = cudaFuncSetAttribute(search_kernel<false, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    search_kernel<false, 512><<<blocks, warps_per_block * 32, smem, s>>>(c);
   } else {
-    search_kernel<false, 768><<<blocks, warps_per_block * 32, 0, s>>>(c);
+    if ((e = cudaFuncSetAttribute(search_kernel<false, 768>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    search_kernel<false, 768><<<blocks, warps_per_block * 32, smem, s>>>(c);
   }
   return cudaGetLastError();
 }

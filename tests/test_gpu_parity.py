@@ -244,6 +244,76 @@ def test_ring_worked_example_on_gpu(gorio):
         ix.close()
 
 
+# ------------------------------------------------------------------ whole index resident: the fast path
+@pytest.mark.parametrize("K,L,W", [(1, 1, 1), (10, 64, 4), (10, 10, 1), (64, 64, 4), (10, 200, 8), (100, 256, 16), (5, 33, 3)])
+@pytest.mark.parametrize("fast", [True, False])
+def test_resident_fast_path_and_general_path_both_match_oracle(gorio, cfg1, K, L, W, fast):
+    """With the whole index preloaded a warp runs each query start to end (list in registers,
+    candidates in shared memory); tuning.no_fast_path sends the same search through the general
+    park-and-resume path.  Both must give the oracle's ids, distances and counters."""
+    w, _ = cfg1
+    q = w.queries[:300]
+    ref = OracleIndex.from_workload(w).search(q, K, L, W, threads=4)
+    got = _gpu_search(gorio, w, w.n_pages, K=K, L=L, W=W, queries=q, preload=True, tuning=dict(no_fast_path=0 if fast else 1))
+    _assert_exact(got, ref)
+    st = got["stats"]
+    assert st["pages_missed"] == 0 and st["pages_fetched"] == 0 and st["queries_done"] == 300
+    assert st["pages_hit"] == int(ref["counters"][:, 3].sum() + ref["counters"][:, 2].sum())      # one lookup per item
+
+
+@pytest.mark.parametrize("tuning", [dict(warps_per_block=2), dict(warps_per_block=5, blocks_per_sm=2), dict(warps_per_block=24),
+                                    dict(max_inflight=7)],
+                         ids=lambda t: "-".join(f"{k}={v}" for k, v in t.items()))
+def test_resident_fast_path_geometry_and_slot_recycling(gorio, cfg1, tuning):
+    """Far more queries than worker warps or query slots (slots are recycled) and odd launch
+    geometries on the fast path.  (Its hash-set form of the visited / page sets is what the
+    allocation-free entry point runs; see test_zz_no_alloc.py.)"""
+    w, ref = cfg1
+    reps = 6
+    q = np.tile(w.queries, (reps, 1))
+    rows = np.arange(q.shape[0]) % w.nq
+    got = _gpu_search(gorio, w, w.n_pages, queries=q, preload=True, tuning=tuning)
+    assert (got["ids"] == ref["ids"][rows]).all() and (got["dists"] == ref["dists"][rows]).all()
+    assert (got["counters"] == ref["counters"][rows]).all() and (got["pages"] == ref["counters"][rows, 0]).all()
+    assert got["stats"]["queries_done"] == q.shape[0]
+
+
+def test_resident_fast_path_other_shapes(gorio):
+    """fp32 vectors (3 blocks of chunks), a PQ index (rerank pool in registers), vectors that are
+    not whole 16-byte chunks (strided path) and 10-per-page records, all fully resident."""
+    from workloads import node_bytes as nbytes
+    w5 = make_config(5, scale=0.005, nq=300)
+    ref5 = OracleIndex.from_workload(w5).search(w5.queries, w5.K, w5.L, w5.W, threads=4)
+    _fp32_parity(w5, _gpu_search(gorio, w5, w5.n_pages, preload=True), ref5)
+    w3 = make_config(3, scale=0.03, nq=400)
+    ref3 = OracleIndex.from_workload(w3).search(w3.queries, w3.K, w3.L, w3.W, threads=4)
+    _assert_exact(_gpu_search(gorio, w3, w3.n_pages, preload=True), ref3)
+    w3.pq_centroids, w3.pq_codes = train_pq(w3.data, m=32, sample=16384, iters=4)
+    for L, W, K in ((50, 1, 10), (100, 8, 10), (64, 4, 28), (64, 4, 40)):      # K + W = 44: the general path takes it
+        refp = OracleIndex.from_workload(w3, use_pq=True).search(w3.queries, K, L, W, threads=4)
+        _assert_exact(_gpu_search(gorio, w3, w3.n_pages, K=K, L=L, W=W, use_pq=True, preload=True), refp)
+    d, R = 20, 12
+    npp = 4096 // nbytes(d, np.uint8, R)
+    wo = make_workload("odd", "u8", 6000, 6, 300, d, R - 4, 4, npp, clustered_knn=True, cross_only=False, K=10, L=48, W=3)
+    refo = OracleIndex.from_workload(wo).search(wo.queries, wo.K, wo.L, wo.W, threads=4)
+    _assert_exact(_gpu_search(gorio, wo, wo.n_pages, preload=True), refo)
+
+
+def test_resident_fast_path_reports_a_corrupt_page(gorio):
+    from helpers import ring_index
+    data, deg, nbrs, pages = ring_index([0, 10, 20, 30], d=4, npp=1)
+    nbrs[1, 1] = 99                                      # neighbour id >= N
+    pages = write_page_store(data, deg, nbrs, 1)
+    ix = gorio.Index(pages, 4, 4, "u8", 2, 1, 0)
+    try:
+        ix.cache_config(16, preload=True)
+        with pytest.raises(gorio.GorioError) as e:
+            ix.search(torch.zeros((3, 4), dtype=torch.uint8).cuda(), 1, 4, 1)
+        assert e.value.status == 7
+    finally:
+        ix.close()
+
+
 # ------------------------------------------------------------------ failure handling without faults
 def test_corrupt_page_is_reported_not_trapped(gorio):
     from helpers import ring_index
