@@ -54,6 +54,69 @@ __device__ __forceinline__ void bitonic_sort(u64 (&x)[NPL], u32 lane, u32 k_firs
   }
 }
 
+// Fold n new keys into the sorted list xl (H keys per lane, ascending, padded beyond len; the list
+// never holds more than L <= 32*H keys).  A chunk of new keys is sorted on its own, descending, so
+// that list ++ chunk is bitonic; one compare-exchange stage then leaves the 32*H smallest of both
+// in xl (everything else could not stay in the list anyway and is dropped on the spot), and one
+// merge pass over H registers re-sorts them.  The chunk's sorting network is picked by its size
+// (32, 64 or 32*H keys): after the first few iterations only a handful of new keys beat the
+// list's worst, and callers pass only those.  GLOBAL: the keys are read with L2 loads from
+// global memory instead of plain loads (shared memory).
+template <int H, bool GLOBAL>
+__device__ __forceinline__ void list_insert(u64 (&xl)[H], u32 &len, const u64 *keys, u32 n, u32 L, u32 lane) {
+  for (u32 done = 0; done < n;) {
+    const u32 take = min(32u * (u32)H, n - done);
+    const u64 *src = keys + done;
+    u64 y[H];
+    if (H > 1 && take <= 32u) {
+      u64 t[1];
+      t[0] = lane < take ? (GLOBAL ? ld_u64(src + lane) : src[lane]) : kPadKey;
+      bitonic_sort<1>(t, lane, 2, true);
+#pragma unroll
+      for (int r = 0; r < H; ++r) y[r] = r == H - 1 ? t[0] : kPadKey;
+    } else if (H > 2 && take <= 64u) {
+      u64 t[2];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const u32 e = (u32)r * 32u + lane;
+        t[r] = e < take ? (GLOBAL ? ld_u64(src + e) : src[e]) : kPadKey;
+      }
+      bitonic_sort<2>(t, lane, 2, true);
+#pragma unroll
+      for (int r = 0; r < H; ++r) y[r] = r == H - 2 ? t[0] : (r == H - 1 ? t[1] : kPadKey);
+    } else {
+#pragma unroll
+      for (int r = 0; r < H; ++r) {
+        const u32 e = (u32)r * 32u + lane;
+        y[r] = e < take ? (GLOBAL ? ld_u64(src + e) : src[e]) : kPadKey;
+      }
+      bitonic_sort<H>(y, lane, 2, true);
+    }
+#pragma unroll
+    for (int r = 0; r < H; ++r) xl[r] = xl[r] < y[r] ? xl[r] : y[r];
+    bitonic_sort<H>(xl, lane, 32u * (u32)H);
+    len = min(L, len + take);
+    done += take;
+#pragma unroll
+    for (int r = 0; r < H; ++r) {
+      const u32 e = (u32)r * 32u + lane;
+      if (e >= len) xl[r] = kPadKey;
+    }
+  }
+}
+
+// The list's L-th key once it is full (what a new key has to beat, with the expanded bit set so
+// that the comparison ignores that bit), all ones before.
+template <int H>
+__device__ __forceinline__ u64 list_worst(const u64 (&xl)[H], u32 len, u32 L, u32 lane) {
+  const u32 wi = L - 1u;
+  u64 worst = kPadKey;
+#pragma unroll
+  for (int r = 0; r < H; ++r)
+    if ((u32)r == wi / 32u) worst = __shfl_sync(0xffffffffu, xl[r], wi % 32u);
+  return len == L ? (worst | 1ull) : kPadKey;
+}
+
 __device__ __forceinline__ void write_result(const Ctx &c, u32 qid, u32 k, u64 key, bool valid) {
   const u64 o = (u64)qid * c.K + k;
   c.out_ids[o] = valid ? key_id(key) : kInvalidId;
@@ -65,90 +128,82 @@ __device__ __forceinline__ void write_result(const Ctx &c, u32 qid, u32 k, u64 k
 // then choose and mark the frontier: the first W unexpanded entries in key order.  The
 // frontier's node ids become the items of the next (PH_EXPAND) batch.  Returns |frontier|;
 // 0 means the search of this query is over (exact mode: the results are written here).
-template <int NPL>
-__device__ __noinline__ u32 merge_select(const Ctx &c, u32 qs, u32 lane) {
+// H: list keys per lane (L <= 32*H).  wk: this warp's candidate area in shared memory (WR keys):
+// only candidates that beat the list's worst key are gathered there and sorted.
+template <int H>
+__device__ __noinline__ u32 merge_select(const Ctx &c, u32 qs, u32 lane, u64 *wk) {
   QHdr *h = c.hdr + qs;
   u32 len = uld(&h->list_len);
   const u32 nc = uld(&h->n_items);
   u64 *list = c.list + (u64)qs * c.L;
   const u64 *cand = c.cand + (u64)qs * c.WR;
-  // The list (sorted, at most L <= 16*NPL keys) lives in the lower half of the registers.  A
-  // chunk of up to 16*NPL new candidates is sorted on its own, descending, in the upper half,
-  // which makes the whole array bitonic; one merge pass then orders it, and everything beyond
-  // L is dropped.  (Sorting list and candidates together cost 2-4x the compare-exchanges.)
-  constexpr int H = NPL / 2;
-  constexpr u32 HALF = 16u * NPL;
-  u64 x[NPL];
+  const u32 lt = (1u << lane) - 1u;
+  u64 xl[H];
 #pragma unroll
-  for (int r = 0; r < NPL; ++r) {
+  for (int r = 0; r < H; ++r) {
     const u32 e = (u32)r * 32u + lane;
-    x[r] = e < len ? ld_u64(list + e) : kPadKey;
+    xl[r] = e < len ? ld_u64(list + e) : kPadKey;
   }
-  u32 done = 0;
-  while (done < nc) {
-    const u32 take = min(HALF, nc - done);
-    u64 y[H];
+  const u64 worst = list_worst<H>(xl, len, c.L, lane);
+  u32 kept = 0;
+  for (u32 base = 0; base < nc; base += 128u) {          // four loads per lane in flight
+    u64 key[4];
 #pragma unroll
-    for (int r = 0; r < H; ++r) {
-      const u32 e = (u32)r * 32u + lane;
-      y[r] = e < take ? ld_u64(cand + done + e) : kPadKey;
+    for (int k = 0; k < 4; ++k) {
+      const u32 i = base + 32u * (u32)k + lane;
+      key[k] = i < nc ? ld_u64(cand + i) : kPadKey;
     }
-    bitonic_sort<H>(y, lane, 2, true);
 #pragma unroll
-    for (int r = 0; r < H; ++r) x[H + r] = y[r];
-    bitonic_sort<NPL>(x, lane, 32u * NPL);
-    len = min(c.L, len + take);
-    done += take;
-#pragma unroll
-    for (int r = 0; r < NPL; ++r) {
-      const u32 e = (u32)r * 32u + lane;
-      if (e >= len) x[r] = kPadKey;
+    for (int k = 0; k < 4; ++k) {
+      const bool keep = key[k] < worst;
+      const u32 b = __ballot_sync(0xffffffffu, keep);
+      if (keep) wk[kept + __popc(b & lt)] = key[k];
+      kept += __popc(b);
     }
   }
+  __syncwarp();
+  list_insert<H, false>(xl, len, wk, kept, c.L, lane);
+  __syncwarp();
   // frontier
   u32 taken = 0;
   u32 *items = c.items + (u64)qs * c.WR;
 #pragma unroll
-  for (int r = 0; r < NPL; ++r) {
+  for (int r = 0; r < H; ++r) {
     const u32 e = (u32)r * 32u + lane;
-    const bool un = e < len && !(x[r] & 1ull);
+    const bool un = e < len && !(xl[r] & 1ull);
     const u32 b = __ballot_sync(0xffffffffu, un);
     if (taken < c.W && b) {
-      const u32 rank = taken + __popc(b & ((1u << lane) - 1u));
-      if (un && rank < c.W) { x[r] |= 1ull; st_u32(items + rank, key_id(x[r])); }
+      const u32 rank = taken + __popc(b & lt);
+      if (un && rank < c.W) { xl[r] |= 1ull; st_u32(items + rank, key_id(xl[r])); }
       taken = min(c.W, taken + (u32)__popc(b));
     }
   }
 #pragma unroll
-  for (int r = 0; r < NPL; ++r) {
+  for (int r = 0; r < H; ++r) {
     const u32 e = (u32)r * 32u + lane;
-    if (e < len) st_u64(list + e, x[r]);
+    if (e < len) st_u64(list + e, xl[r]);
   }
   if (lane == 0) st_u32(&h->list_len, len);
   {   // the L-th key once the list is full: what a new candidate has to beat
-    const u32 wi = c.L - 1u;
-    u64 worst = kPadKey;
-#pragma unroll
-    for (int r = 0; r < NPL; ++r)
-      if ((u32)r == wi / 32u) worst = __shfl_sync(0xffffffffu, x[r], wi % 32u);
-    if (lane == 0) st_u64((u64 *)&h->worst_lo, len == c.L ? (worst | 1ull) : kPadKey);
+    const u64 w2 = list_worst<H>(xl, len, c.L, lane);
+    if (lane == 0) st_u64((u64 *)&h->worst_lo, w2);
   }
   if (taken == 0 && c.pq_m == 0) {
     const u32 qid = uld(&h->qid);
 #pragma unroll
-    for (int r = 0; r < NPL; ++r) {
+    for (int r = 0; r < H; ++r) {
       const u32 e = (u32)r * 32u + lane;
-      if (e < c.K) write_result(c, qid, e, x[r], e < len);
+      if (e < c.K) write_result(c, qid, e, xl[r], e < len);
     }
   }
   return taken;
 }
 
-__device__ u32 merge_select_dispatch(const Ctx &c, u32 qs, u32 lane) {
-  if (c.L <= 32) return merge_select<2>(c, qs, lane);        // the list fits half of 32*NPL keys
-  if (c.L <= 64) return merge_select<4>(c, qs, lane);
-  if (c.L <= 128) return merge_select<8>(c, qs, lane);
-  return merge_select<16>(c, qs, lane);
+__device__ u32 merge_select_dispatch(const Ctx &c, u32 qs, u32 lane, u64 *wk) {
+  if (c.L <= 32) return merge_select<1>(c, qs, lane, wk);
+  if (c.L <= 64) return merge_select<2>(c, qs, lane, wk);
+  if (c.L <= 128) return merge_select<4>(c, qs, lane, wk);
+  return merge_select<8>(c, qs, lane, wk);
 }
 
 // PQ mode: fold the exact distances of the nodes just expanded into the rerank pool

@@ -100,17 +100,34 @@ __device__ __noinline__ void build_lut(const Ctx &c, u32 qid, u32 *lut, u32 lane
     default: build_lut_gen<4>(c, q, lut, lane); break;
   }
 }
-// One node per lane: the lane reads the node's code (pq_m bytes, 4 at a time) and sums pq_m
-// independent table entries from shared memory -- no cross-lane reduction, 32 nodes per pass.
+// One node per lane: the lane reads the node's code (pq_m bytes) and sums pq_m independent table
+// entries from shared memory -- no cross-lane reduction, 32 nodes per pass.  The code is read in
+// 16-byte chunks, the next chunk's load issued before the current one is looked up, so a 32-byte
+// code costs one round trip to L2/HBM, not one per word; the loop body (16 lookups) is kept
+// rolled to stay small in the instruction cache.
+__device__ __forceinline__ u32 adc_word(const u16 *lo, const u32 *hi, u32 sub0, u32 cw) {
+  return lut_get(lo, hi, ((sub0 + 0u) << 8) + (cw & 255u)) + lut_get(lo, hi, ((sub0 + 1u) << 8) + ((cw >> 8) & 255u)) +
+         lut_get(lo, hi, ((sub0 + 2u) << 8) + ((cw >> 16) & 255u)) + lut_get(lo, hi, ((sub0 + 3u) << 8) + (cw >> 24));
+}
 __device__ __forceinline__ u32 lane_adc(const Ctx &c, const u32 *lut, u32 v) {
-  const u32 *code = (const u32 *)(c.pq_codes + (u64)v * c.pq_m);
+  const u8 *code = c.pq_codes + (u64)v * c.pq_m;
   const u16 *lo = (const u16 *)lut;
   const u32 *hi = lut_hi(c, lut);
   u32 acc = 0;
-  for (u32 w = 0; w < (c.pq_m >> 2); ++w) {
-    const u32 cw = __ldg(code + w);
-    acc += lut_get(lo, hi, ((4u * w + 0u) << 8) + (cw & 255u)) + lut_get(lo, hi, ((4u * w + 1u) << 8) + ((cw >> 8) & 255u)) +
-           lut_get(lo, hi, ((4u * w + 2u) << 8) + ((cw >> 16) & 255u)) + lut_get(lo, hi, ((4u * w + 3u) << 8) + (cw >> 24));
+  if ((c.pq_m & 15u) == 0u && ((uintptr_t)c.pq_codes & 15u) == 0u) {
+    const uint4 *c4 = (const uint4 *)code;
+    const u32 nch = c.pq_m >> 4;
+    uint4 cur = __ldg(c4);
+#pragma unroll 1
+    for (u32 ch = 0; ch < nch; ++ch) {
+      uint4 nxt = cur;
+      if (ch + 1u < nch) nxt = __ldg(c4 + ch + 1u);
+      acc += adc_word(lo, hi, 16u * ch, cur.x) + adc_word(lo, hi, 16u * ch + 4u, cur.y) +
+             adc_word(lo, hi, 16u * ch + 8u, cur.z) + adc_word(lo, hi, 16u * ch + 12u, cur.w);
+      cur = nxt;
+    }
+  } else {
+    for (u32 w = 0; w < (c.pq_m >> 2); ++w) acc += adc_word(lo, hi, 4u * w, __ldg((const u32 *)code + w));
   }
   return acc;
 }

@@ -114,7 +114,7 @@ __device__ __noinline__ bool wait_in_place(const Ctx &c, u32 qs, u32 lane) {
 // lut_qid: the query whose table currently sits in this warp's shared memory (kept across calls,
 // so a query that runs several phases in a row on one warp builds its table once).
 template <bool PQ>
-__device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut, u32 &lut_qid) {
+__device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut, u32 &lut_qid, u32 *ws) {
   QHdr *h = c.hdr + qs;
   u64 tp = c.prof ? globaltimer() : 0;
   for (u32 guard = 0; guard < 4u * c.max_iters + 64u; ++guard) {
@@ -140,7 +140,7 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut, u32 &lut_qid
         if (!go && !(c.blocking && wait_in_place<PQ>(c, qs, lane))) return;
       }
     } else if (phase == PH_EVAL) {
-      const u32 nf = merge_select_dispatch(c, qs, lane);
+      const u32 nf = merge_select_dispatch(c, qs, lane, (u64 *)ws);
       phase_mark(c, tp, S_P_MERGE, lane);
       if (nf == 0) {
         finish_query(c, qs, lane);
@@ -333,9 +333,9 @@ __global__ void __launch_bounds__(MAXT, 1) search_kernel(const Ctx c) {
   const u32 lane = lane_id(), warp = threadIdx.x >> 5;
   if (blockIdx.x == 0 && warp == 0) { poller(c, lane); return; }
   u32 *lut = PQ ? smem_lut + (u64)warp * c.pq_m * kPqLutWords : nullptr;
+  // this warp's candidate area (WR keys and 16 frontier ids), behind the PQ tables
+  u32 *ws = smem_lut + (PQ ? (u64)(blockDim.x >> 5) * c.pq_m * kPqLutWords : 0) + (u64)warp * resident_warp_words(c.WR);
   if (c.resident_fast) {                   // whole index resident: queries run start to end on one warp
-    const u32 n_warps = blockDim.x >> 5;
-    u32 *ws = smem_lut + (PQ ? (u64)n_warps * c.pq_m * kPqLutWords : 0) + (u64)warp * resident_warp_words(c.WR);
     resident_worker<PQ>(c, lane, lut, ws);
     return;
   }
@@ -375,7 +375,7 @@ __global__ void __launch_bounds__(MAXT, 1) search_kernel(const Ctx c) {
       continue;
     }
     if (warp_pop(c, c.run, v, lane)) {
-      run_query<PQ>(c, v, lane, lut, lut_qid); idle = 0;
+      run_query<PQ>(c, v, lane, lut, lut_qid, ws); idle = 0;
       const u64 t = globaltimer(); t_run += t - tp; tp = t; ++n_run;
       continue;
     }

@@ -511,10 +511,10 @@ int launch_geometry(gorio_index *ix, u32 nq, u32 K, u32 W, u32 *blocks_out, u32 
     auto_warps = auto_warps < 8u ? 8u : (auto_warps > 24u ? 24u : auto_warps);
     if (g.resident_fast && auto_warps > 16u) auto_warps = 16u;     // the fast path wants the 128-register build
   }
-  u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? (g.resident_fast ? 12u : 10u) : auto_warps);
+  u32 warps = ix->tune.warps_per_block ? ix->tune.warps_per_block : (pq ? 10u : auto_warps);
   const size_t per_warp = search_smem_per_warp(g);
-  if (per_warp) {                 // per-warp tables / candidate areas in shared memory
-    u32 lim = (u32)((220u * 1024u) / per_warp);
+  if (per_warp) {                 // per-warp tables / candidate areas in shared memory (227 KB per block at most)
+    u32 lim = (u32)((227u * 1024u) / per_warp);
     if (pq && lim > 12u) lim = 12u;      // the PQ kernel is built for at most 12 warps
     if (warps > lim) warps = lim;
   }

@@ -94,10 +94,9 @@ cudaError_t launch_cache_reset(const Ctx &c, u32 preloaded, cudaStream_t s) {
   return cudaGetLastError();
 }
 
-// Dynamic shared memory per warp: the PQ distance table, and on the resident fast path the
-// warp's candidate area.
+// Dynamic shared memory per warp: the PQ distance table and the warp's candidate area.
 size_t search_smem_per_warp(const Ctx &c) {
-  return (c.pq_m ? (size_t)c.pq_m * kPqLutWords * 4 : 0) + (c.resident_fast ? (size_t)resident_warp_words(c.WR) * 4 : 0);
+  return (c.pq_m ? (size_t)c.pq_m * kPqLutWords * 4 : 0) + (size_t)resident_warp_words(c.WR) * 4;
 }
 
 template <typename K>
