@@ -131,11 +131,11 @@ __device__ __noinline__ void resident_query(const Ctx &c, u32 qs, u32 qid, u32 l
     // into shared memory; four neighbour positions per lane in flight
     out = 0;
     const u32 total = taken * c.R;
-    for (u32 base = 0; base < total; base += 128u) {
-      u32 v[4], dg[4], pos[4];
-      bool ok[4];
+    for (u32 base = 0; base < total; base += 256u) {
+      u32 v[8], dg[8], pos[8];
+      bool ok[8];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
+      for (int k = 0; k < 8; ++k) {
         const u32 p = base + 32u * (u32)k + lane;
         ok[k] = p < total;
         const u32 f = ok[k] ? p / c.R : 0u;
@@ -145,15 +145,15 @@ __device__ __noinline__ void resident_query(const Ctx &c, u32 qs, u32 qid, u32 l
         dg[k] = ok[k] ? __ldcg(adj) : 0u;
         v[k] = ok[k] ? __ldcg(adj + 1 + pos[k]) : kInvalidId;
       }
-      // all four insertions in flight before any result is looked at
-      u32 r[4];
+      // all eight insertions in flight before any result is looked at
+      u32 r[8];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
+      for (int k = 0; k < 8; ++k) {
         r[k] = 3u;                                           // not a neighbour position
         if (ok[k] && dg[k] <= c.R && pos[k] < dg[k]) r[k] = v[k] < c.n_nodes ? qset_insert(seen, c.seen_cap, seen_bm, v[k]) : 4u;
       }
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
+      for (int k = 0; k < 8; ++k) {
         if (ok[k] && pos[k] == 0u) {                         // one lane per expanded node
           if (dg[k] > c.R) raise(c, 7, 0x91, qs, dg[k]); else my_deg += dg[k];
         }
