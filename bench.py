@@ -207,6 +207,7 @@ def main():
     ap.add_argument("--no-parity", action="store_true", help="skip the oracle comparison of the timed outputs")
     ap.add_argument("--warps", type=int, default=0, help="warps per block of the persistent kernel (0 = the library's choice)")
     ap.add_argument("--no-fast-path", action="store_true", help="whole index resident: use the general path anyway")
+    ap.add_argument("--timeout-ms", type=int, default=120_000, help="bound on one search call (profiling captures use a short one)")
     ap.add_argument("--L", type=int, default=None)
     ap.add_argument("--W", type=int, default=None)
     args = ap.parse_args()
@@ -289,7 +290,7 @@ def main():
 
     def reset_cache():
         ix.cache_config(state["cap"], remote_latency_ns=state["lat_ns"], max_outstanding=state["max_out"],
-                        preload=state["preload"], timeout_ms=120_000, granularity=args.granularity,
+                        preload=state["preload"], timeout_ms=args.timeout_ms, granularity=args.granularity,
                         copy_engine=args.copy_engine)
         ix.stats_reset()
         l2_flush(flush)
