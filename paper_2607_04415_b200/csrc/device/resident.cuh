@@ -128,7 +128,7 @@ __device__ __noinline__ void resident_query(const Ctx &c, u32 qs, u32 qid, u32 l
     }
 
     // adjacency lists straight from the pages, through the exact visited set, survivors compacted
-    // into shared memory; four neighbour positions per lane in flight
+    // into shared memory; eight neighbour positions per lane in flight
     out = 0;
     const u32 total = taken * c.R;
     for (u32 base = 0; base < total; base += 256u) {

@@ -665,8 +665,10 @@ def test_randomized_configurations_match_oracle(gorio, seed):
     tuning = dict(warps_per_block=int(rng.integers(2, 17)), max_inflight=int(rng.choice([0, 8, 64])),
                   stash_entries=int(rng.choice([0, 1, 64, 256])), blocking=int(rng.integers(0, 2)),
                   request_backlog=int(rng.choice([0, 1, 16, 4096])))
-    got = _gpu_search(gorio, w, cap, K=K, L=L, W=W, tuning=tuning, preload=bool(rng.integers(0, 4) == 0),
-                      remote_latency_ns=int(rng.choice([0, 2000, 20000])), max_outstanding=int(rng.choice([1, 8, 256])))
+    preload, lat, depth = bool(rng.integers(0, 4) == 0), int(rng.choice([0, 2000, 20000])), int(rng.choice([1, 8, 256]))
+    copy_engine, gran = bool(rng.integers(0, 4) == 0), str(rng.choice(["page", "page", "record"]))
+    got = _gpu_search(gorio, w, cap, K=K, L=L, W=W, tuning=tuning, preload=preload and gran == "page",
+                      remote_latency_ns=lat, max_outstanding=depth, copy_engine=copy_engine, granularity=gran)
     _assert_exact(got, ref)
     assert got["stats"]["queries_done"] == nq
 
