@@ -11,7 +11,7 @@ LIB_PATH = os.path.join(_HERE, "libgorio.so")
 SOURCES = ["gorio_api.cu", "search_kernels.cu", "noalloc_entry.cu"]
 HEADERS = ["gorio_internal.h", os.path.join("..", "..", "include", "gorio.h")] + [
     os.path.join("device", f) for f in ("mem.cuh", "queue.cuh", "page_cache.cuh", "scoring.cuh", "arrival.cuh", "batch.cuh",
-                                        "list.cuh", "pq.cuh", "scheduler.cuh")]
+                                        "list.cuh", "pq.cuh", "scheduler.cuh", "resident.cuh")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-pthread"]
 
