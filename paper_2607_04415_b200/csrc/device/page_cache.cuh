@@ -44,19 +44,25 @@ __device__ __forceinline__ const u8 *rec_ptr(const Ctx &c, u32 slot, u32 node) {
 
 struct LaneStats { u32 hit, missed, joins, evict, retry, posted; };
 
-// Post a request descriptor: one 64-bit word [page:32][slot:24][lap:8] in host-mapped memory.
-// The ring holds at least twice as many entries as there are slots, and every pending
-// request owns a distinct FILLING slot, so an entry is never overwritten before the proxy
-// has consumed it.  (Section 3.2: reserve a descriptor slot atomically, record page id and
-// target cache slot, publish through a ready flag -- here the lap tag inside the word.)
+// Post a request descriptor: one 64-bit word [page:32][slot:24][lap:8].  The ring holds at least
+// twice as many entries as there are slots, and every pending request owns a distinct FILLING
+// slot, so an entry is never overwritten before it has been consumed.  (Section 3.2: reserve a
+// descriptor slot atomically, record page id and target cache slot, publish through a ready flag
+// -- here the lap tag inside the word.)
+// The worker writes the descriptor into the DEVICE copy of the ring only; the poster warp forwards
+// it to the host-visible ring (see poster()).  Worker warps therefore never have a store to host
+// memory in flight behind a post: every later fence of such a warp would have to wait for it, and
+// with the host link saturated by page reads that wait was ~5 us per fence and 18 us for the
+// system-scope fence that used to stand here.  A posted request waits in the ring for its turn
+// in the proxy's window anyway (the backlog is several windows deep), so the microsecond the
+// forwarding adds costs nothing.
 __device__ __forceinline__ void post_request(const Ctx &c, u32 page, u32 slot) {
   const u32 idx = atomicAdd(&c.ctl->ring_head, 1u);
   atomicAdd(&c.cs->in_flight, 1);
   const u32 lap = ((idx >> c.ring_shift) % 255u) + 1u;
   const u64 e = ((u64)page << 32) | ((u64)slot << 8) | lap;
-  st_u64(c.ring_dev + (idx & c.ring_mask), e);   // device copy: what copy and arrival tickets refer to
-  __threadfence_system();      // page word, slot label and device copy before the host can act
-  st_sys_u64(c.ring + (idx & c.ring_mask), e);
+  __threadfence();             // page word and slot label before the descriptor can be seen
+  st_u64(c.ring_dev + (idx & c.ring_mask), e);   // also what copy and arrival tickets refer to
 }
 
 // Requests posted and not yet arrived are kept near a small multiple of the proxy's window:

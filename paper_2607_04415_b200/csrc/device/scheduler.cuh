@@ -308,6 +308,30 @@ __device__ void poller(const Ctx &c, u32 lane) {
   if (lane == 0) c.ctl->stats[S_POLLS] = it;
 }
 
+// Warp 1 of block 0 forwards request descriptors from the device copy of the ring to the
+// host-visible ring, in ring order, up to 32 per look (lane i looks at entry next + i; the ready
+// ones form a prefix as far as this look is concerned).  It is the only warp that writes
+// descriptors to host memory.
+__device__ void poster(const Ctx &c, u32 lane) {
+  u32 next = 0, it = 0;
+  const u64 t0 = globaltimer();
+  for (;;) {
+    const u32 idx = next + lane;
+    const u64 e = ld_u64(c.ring_dev + (idx & c.ring_mask));
+    const bool ready = (u32)(e & 0xFFu) == ((idx >> c.ring_shift) % 255u) + 1u;
+    const u32 n = (u32)__ffs((int)~__ballot_sync(0xffffffffu, ready)) - 1u;      // leading ready entries (32 if all)
+    const u32 cnt = n > 32u ? 32u : n;
+    if (lane < cnt) st_sys_u64(c.ring + (idx & c.ring_mask), e);
+    next += cnt;
+    if (cnt == 0) {
+      if (warp_stopped(c)) break;
+      __nanosleep(200);
+      u32 late = ((++it & 1023u) == 0 && globaltimer() - t0 > c.timeout_ns) ? 1u : 0u;
+      if (__shfl_sync(0xffffffffu, late, 0)) { if (lane == 0) raise(c, 5, 0xB4); break; }
+    }
+  }
+}
+
 // Take one ticket from a (count, head) pair released by the poller; lane 0 only.
 __device__ __forceinline__ bool take_ticket(int *count, u32 *head, u32 &idx) {
   if ((int)ld_u32((const u32 *)count) <= 0) return false;
@@ -332,6 +356,7 @@ __global__ void __launch_bounds__(MAXT, 1) search_kernel(const Ctx c) {
   extern __shared__ u32 smem_lut[];
   const u32 lane = lane_id(), warp = threadIdx.x >> 5;
   if (blockIdx.x == 0 && warp == 0) { poller(c, lane); return; }
+  if (blockIdx.x == 0 && warp == 1 && !c.identity) { poster(c, lane); return; }     // (nothing is ever posted when the whole index is resident)
   u32 *lut = PQ ? smem_lut + (u64)warp * c.pq_m * kPqLutWords : nullptr;
   // this warp's candidate area (WR keys and 16 frontier ids), behind the PQ tables
   u32 *ws = smem_lut + (PQ ? (u64)(blockDim.x >> 5) * c.pq_m * kPqLutWords : 0) + (u64)warp * resident_warp_words(c.WR);

@@ -480,6 +480,7 @@ void fill_ctx(gorio_index *ix, const void *queries_dev, u32 nq, u32 K, u32 L, u3
   c.max_iters = 64u * L + 1024u;
   c.blocking = ix->tune.blocking ? 1u : 0u;
   c.idle_ns = 8000u;
+  { const char *e = std::getenv("GORIO_IDLE_NS"); if (e) c.idle_ns = (u32)std::atoi(e); }      // debug aid
   // default backlog: 4 x the proxy's window, but no more than 1024 (about what keeps the host
   // link busy) unless the window itself is larger
   c.max_in_flight = ix->tune.request_backlog ? ix->tune.request_backlog
@@ -518,7 +519,7 @@ int launch_geometry(gorio_index *ix, u32 nq, u32 K, u32 W, u32 *blocks_out, u32 
     if (pq && lim > 12u) lim = 12u;      // the PQ kernel is built for at most 12 warps
     if (warps > lim) warps = lim;
   }
-  if (warps < 2) return fail(ix, GORIO_ERR_INVALID_ARG, "search: need at least 2 warps per block (the poller and a worker)");
+  if (warps < 2) return fail(ix, GORIO_ERR_INVALID_ARG, "search: need at least 2 warps per block (block 0 gives two to the poller and the poster)");
   int occ = 0;
   CK(search_occupancy(g, warps, &occ));
   if (occ < 1) return fail(ix, GORIO_ERR_INVALID_ARG, "search: launch geometry does not fit an SM");
@@ -742,6 +743,7 @@ int gorio_search(gorio_index *ix, const void *queries_dev, uint32_t nq, uint32_t
   flush_wc();
   std::atomic_thread_fence(std::memory_order_seq_cst);
 
+  CK(cudaMemsetAsync(c.ring_dev, 0, (size_t)ix->ring_cap * 8, stream));      // no descriptor of an earlier search may look ready
   CK(cudaMemsetAsync(c.seen, c.seen_bitmap ? 0x00 : 0xFF, (size_t)c.n_qslots * c.seen_cap * 4, stream));
   CK(cudaMemsetAsync(c.pset, c.pset_bitmap ? 0x00 : 0xFF, (size_t)c.n_qslots * c.pset_cap * 4, stream));
   if (c.stash_cap) CK(cudaMemsetAsync(c.stash_tag, 0xFF, (size_t)c.n_qslots * c.stash_cap * 4, stream));

@@ -13,7 +13,8 @@
 //                        score them from resident PQ codes (PQ mode)
 // "Issuing" a batch of page items means, per item: look the page up in the cache; on a hit
 // consume it now; if the page is in flight register as a waiter; if it is absent claim a
-// slot (clock eviction), post a request descriptor to the host-visible ring and register.
+// slot (clock eviction), post a request descriptor (the poster warp forwards it to the
+// host-visible ring) and register.
 // A page that arrives is consumed for every registered waiter by whichever warp picks the
 // arrival up, using only the waiter's query vector, so no page stays pinned for a query.
 // The last item consumed of a batch pushes the query back onto the runnable queue.
