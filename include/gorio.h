@@ -112,9 +112,10 @@ typedef struct {
  * and then mark its ready entry, and Section 4 calls the CPU side a transport proxy.  Here the
  * default is GORIO_COPY_SM_PULL, and GORIO_COPY_ENGINE is the literal reading kept as an option.
  * The reason is the request rate: the benchmark configuration needs about 11 million 4 KB fills
- * per second, a cudaMemcpyAsync costs the calling thread about 2 microseconds (0.5 million per
- * second and thread), and no batched-copy runtime call is usable on the target machines; SM
- * reads of pinned memory reach 51.5 of the 55.5 GB/s a bulk copy gets on the same link.  In both
+ * per second; a small cudaMemcpyAsync issued while the persistent kernel is resident completes about
+ * a millisecond after the call (0.23 million fills per second with 256 in flight) and costs the
+ * calling thread about 2 microseconds, and no batched-copy runtime call is usable on the target
+ * machines; SM reads of pinned memory reach 51.5 of the 55.5 GB/s a bulk copy gets on the same link.  In both
  * modes the proxy alone admits requests, bounds the number outstanding, applies the latency and
  * publishes completions in ring order, and it never looks at search state.
  * Calling gorio_cache_config again re-creates an empty (or preloaded) cache.
