@@ -215,6 +215,8 @@ def main():
                          "sliced across the ranks, results gathered and checked on rank 0")
     ap.add_argument("--no-parity", action="store_true", help="skip the oracle comparison of the timed outputs")
     ap.add_argument("--warps", type=int, default=0, help="warps per block of the persistent kernel (0 = the library's choice)")
+    ap.add_argument("--visited-capacity", type=int, default=0,
+                    help="entries of the per-query visited set (0 = the library's default; a bitmap is used when it is no larger)")
     ap.add_argument("--no-fast-path", action="store_true", help="whole index resident: use the general path anyway")
     ap.add_argument("--timeout-ms", type=int, default=120_000, help="bound on one search call (profiling captures use a short one)")
     ap.add_argument("--L", type=int, default=None)
@@ -285,7 +287,8 @@ def main():
     use_pq = args.config == 4
     ix = g.Index.from_workload(w, device=local, use_pq=use_pq)
     if args.blocking or args.warps or args.no_fast_path:
-        ix.set_tuning(blocking=int(args.blocking), warps_per_block=args.warps, no_fast_path=int(args.no_fast_path))
+        ix.set_tuning(blocking=int(args.blocking), warps_per_block=args.warps, no_fast_path=int(args.no_fast_path),
+                      visited_capacity=args.visited_capacity)
     q_dev = torch.as_tensor(my_q).to(dev)
     q_pin = torch.as_tensor(my_q).pin_memory()
     outs_pin = dict(ids=torch.empty((my_nq, w.K), dtype=torch.int32).pin_memory(),
