@@ -217,6 +217,8 @@ def main():
     ap.add_argument("--warps", type=int, default=0, help="warps per block of the persistent kernel (0 = the library's choice)")
     ap.add_argument("--visited-capacity", type=int, default=0,
                     help="entries of the per-query visited set (0 = the library's default; a bitmap is used when it is no larger)")
+    ap.add_argument("--shared-pull", action="store_true",
+                    help="ablation: worker warps pull admitted pages between their other work (no dedicated puller warps)")
     ap.add_argument("--no-fast-path", action="store_true", help="whole index resident: use the general path anyway")
     ap.add_argument("--timeout-ms", type=int, default=120_000, help="bound on one search call (profiling captures use a short one)")
     ap.add_argument("--L", type=int, default=None)
@@ -286,9 +288,9 @@ def main():
     lat_ns, max_out = int(w.latency_us * 1000), w.max_outstanding
     use_pq = args.config == 4
     ix = g.Index.from_workload(w, device=local, use_pq=use_pq)
-    if args.blocking or args.warps or args.no_fast_path:
+    if args.blocking or args.warps or args.no_fast_path or args.shared_pull or args.visited_capacity:
         ix.set_tuning(blocking=int(args.blocking), warps_per_block=args.warps, no_fast_path=int(args.no_fast_path),
-                      visited_capacity=args.visited_capacity)
+                      visited_capacity=args.visited_capacity, shared_pull=int(args.shared_pull))
     q_dev = torch.as_tensor(my_q).to(dev)
     q_pin = torch.as_tensor(my_q).pin_memory()
     outs_pin = dict(ids=torch.empty((my_nq, w.K), dtype=torch.int32).pin_memory(),
@@ -426,6 +428,9 @@ def main():
         if i:
             e2e_times.append(float(tt))
     h2d = max(h2d, measure_h2d_gbs(dev, w.pages))     # measured before and after the timed steps; the better one is the peak
+    # what the link gives SM warps that pull scattered 4 KB pages of this store and do nothing else
+    # (the loads of a page fill, as many pages in flight as the window allows): context for the link term
+    sm_pull_gbs = max(ix.link_probe(200_000, max(4, min(int(max_out), 16384))) for _ in range(3))
     ms = statistics.mean(times)
     st = stats_list[len(stats_list) // 2]
     fetched = statistics.mean(s["pages_fetched"] for s in stats_list)
@@ -480,7 +485,9 @@ def main():
             "traffic": None, "peak_kind": f"hbm {pk_kind}; host link measured in this run ({h2d:.1f} GB/s)",
             "terms_ms": {k: 1e3 * v for k, v in terms.items()},
             "pages_fetched": fetched, "fetched_bytes": fetched_bytes, "algorithmic_hbm_bytes": b_hbm,
-            "hbm_achieved_gbs": b_hbm / (ms * 1e-3) / 1e9, "hbm_peak_gbs": pk["hbm_gbs"]}
+            "hbm_achieved_gbs": b_hbm / (ms * 1e-3) / 1e9, "hbm_peak_gbs": pk["hbm_gbs"],
+            "host_link_bulk_copy_gbs": h2d, "host_link_sm_page_pull_gbs": sm_pull_gbs,
+            "fetched_gbs": fetched_bytes / (ms * 1e-3) / 1e9}
     if default_workload:
         # DRAM bytes of one search_kernel launch from a single-pass ncu capture of this command, valid
         # only for the device code it was captured on

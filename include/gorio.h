@@ -100,7 +100,8 @@ typedef struct {
  *                    change.  preload must be 0 in this mode.
  *   copy_mode        who moves a page's bytes from the pinned store into its slot:
  *                    GORIO_COPY_SM_PULL (0, default): the proxy admits the request by advancing a
- *                    counter in host-mapped memory; warps of the search kernel pull the page over
+ *                    counter in host-mapped memory; warps of the search kernel (one puller warp
+ *                    per block, in ring order; see gorio_tuning.shared_pull) pull the page over
  *                    the host link and acknowledge; the proxy publishes the completion after the
  *                    latency.  The proxy makes no CUDA call while a search runs.
  *                    GORIO_COPY_ENGINE (1): the proxy thread itself copies the page, one
@@ -115,7 +116,7 @@ typedef struct {
  * per second; a small cudaMemcpyAsync issued while the persistent kernel is resident completes about
  * a millisecond after the call (0.23 million fills per second with 256 in flight) and costs the
  * calling thread about 2 microseconds, and no batched-copy runtime call is usable on the target
- * machines; SM reads of pinned memory reach 51.5 of the 55.5 GB/s a bulk copy gets on the same link.  In both
+ * machines; SM reads of pinned memory reach 51 of the 55.5 GB/s a bulk copy gets on the same link.  In both
  * modes the proxy alone admits requests, bounds the number outstanding, applies the latency and
  * publishes completions in ring order, and it never looks at search state.
  * Calling gorio_cache_config again re-creates an empty (or preloaded) cache.
@@ -154,6 +155,13 @@ enum { GORIO_GRAN_PAGE = 0, GORIO_GRAN_RECORD = 1 };
  *                    to output without parking it, with the list in registers and the candidates
  *                    in shared memory; with this flag such a search goes through the general
  *                    park-and-resume machinery instead.  Results are identical; for comparisons.
+ *   shared_pull      1 = ablation: no dedicated puller warps.  By default (page granularity, SM
+ *                    pull) the last warp of every block does nothing but pull admitted pages, in
+ *                    ring order: it claims the next request index ahead of time, waits until the
+ *                    admission is known on the GPU and issues the page's reads at once; worker
+ *                    warps pull nothing.  With this flag, as always at record granularity, worker
+ *                    warps take the pulls between their other work (whoever looks first), which
+ *                    starts them later and out of order.  Results are identical.
  *   blocking         1 = ablation: a warp that misses keeps its query and waits in place for
  *                    the pages (the demand-paging baseline of Section 5.1) instead of parking
  *                    the query and taking another; results are identical, only slower.
@@ -167,6 +175,7 @@ typedef struct {
   uint32_t blocking;
   uint32_t request_backlog;
   uint32_t no_fast_path;
+  uint32_t shared_pull;
 } gorio_tuning;
 
 /*
@@ -262,6 +271,22 @@ int gorio_search_host(gorio_index *ix, const void *queries_host, uint32_t nq, ui
 int gorio_stats(gorio_index *ix, gorio_stats_t *out);
 /* Zero every counter of gorio_stats_t (device and proxy side).  No counterpart in the paper. */
 int gorio_stats_reset(gorio_index *ix);
+
+/*
+ * Measurement aid (no counterpart in the paper): what the host link delivers to the access pattern
+ * of a page fill and nothing else.  `pages_in_flight` warps (rounded up to a multiple of four, at
+ * most 16384) each pull whole 4 KB pages of the index's pinned page store into a 4 KB HBM area of
+ * their own, one page at a time with the page's loads all in flight -- the loads a fill of the
+ * search kernel issues -- until `n_pulls` pages have been pulled; pull i reads page hash(i) mod
+ * n_pages (uniformly scattered) or, with `sequential` != 0, page i mod n_pages.  No cache, no proxy,
+ * no latency, no window.  `gbs_out` (HOST) receives n_pulls * 4096 bytes over the kernel's duration
+ * (CUDA events on `cuda_stream`), in GB/s.  bench.py reports it beside the bulk-copy figure: random
+ * 4 KB reads of a store much larger than the host's last-level cache run slower than one long copy.
+ * Allocates and frees its scratch (pages_in_flight x 4 KB) inside the call; blocking; must not
+ * overlap a search on the same index.  Errors: INVALID_ARG, CUDA.
+ */
+int gorio_link_probe(gorio_index *ix, uint32_t n_pulls, uint32_t pages_in_flight, int sequential, void *cuda_stream,
+                     double *gbs_out);
 
 /* Stops the proxy thread, frees every device and host resource of the index, un-pins the page
  * store if the library pinned it.  The handle is invalid afterwards.  (Resource management: no

@@ -14,7 +14,7 @@ _LIB = None
 EXPORTED_SYMBOLS = [
     "gorio_index_open", "gorio_cache_config", "gorio_set_tuning", "gorio_search", "gorio_search_host",
     "gorio_stats", "gorio_stats_reset", "gorio_index_close", "gorio_status_str", "gorio_last_error",
-    "gorio_search_resident_noalloc",
+    "gorio_search_resident_noalloc", "gorio_link_probe",
 ]
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "CUDA", 3: "NOMEM", 4: "STATE", 5: "TIMEOUT",
@@ -46,7 +46,8 @@ class _Tuning(ctypes.Structure):
     _fields_ = [("max_inflight", ctypes.c_uint32), ("visited_capacity", ctypes.c_uint32),
                 ("warps_per_block", ctypes.c_uint32), ("blocks_per_sm", ctypes.c_uint32),
                 ("stash_entries", ctypes.c_uint32), ("blocking", ctypes.c_uint32),
-                ("request_backlog", ctypes.c_uint32), ("no_fast_path", ctypes.c_uint32)]
+                ("request_backlog", ctypes.c_uint32), ("no_fast_path", ctypes.c_uint32),
+                ("shared_pull", ctypes.c_uint32)]
 
 
 _STAT_FIELDS = ["pages_hit", "pages_missed", "pages_fetched", "dedupe_joins", "evictions", "retries",
@@ -87,6 +88,7 @@ def load_library():
     lib.gorio_search_resident_noalloc.argtypes = [ctypes.POINTER(_IndexDesc), vp, vp, u32, u32, u32, u32, vp, vp, vp, vp]
     lib.gorio_stats.argtypes = [vp, ctypes.POINTER(Stats)]
     lib.gorio_stats_reset.argtypes = [vp]
+    lib.gorio_link_probe.argtypes = [vp, u32, u32, ctypes.c_int, vp, ctypes.POINTER(ctypes.c_double)]
     lib.gorio_index_close.argtypes = [vp]
     lib.gorio_status_str.argtypes = [ctypes.c_int]
     lib.gorio_status_str.restype = ctypes.c_char_p
@@ -198,9 +200,9 @@ class Index:
         self._check(self._lib.gorio_cache_config(self._h, ctypes.byref(cfg)))
 
     def set_tuning(self, max_inflight=0, visited_capacity=0, warps_per_block=0, blocks_per_sm=0, stash_entries=0,
-                   blocking=0, request_backlog=0, no_fast_path=0):
+                   blocking=0, request_backlog=0, no_fast_path=0, shared_pull=0):
         t = _Tuning(max_inflight, visited_capacity, warps_per_block, blocks_per_sm, stash_entries, int(blocking),
-                    request_backlog, int(no_fast_path))
+                    request_backlog, int(no_fast_path), int(shared_pull))
         self._check(self._lib.gorio_set_tuning(self._h, ctypes.byref(t)))
 
     def search(self, queries: torch.Tensor, K: int, L: int, W: int, want_counters=True, stream=None):
@@ -242,6 +244,13 @@ class Index:
 
     def stats_reset(self):
         self._check(self._lib.gorio_stats_reset(self._h))
+
+    def link_probe(self, n_pulls: int, pages_in_flight: int, sequential: bool = False, stream=None) -> float:
+        """GB/s the host link delivers to `pages_in_flight` warps pulling 4 KB pages of the store (no search)."""
+        gbs = ctypes.c_double(0.0)
+        sp = ctypes.c_void_p(stream.cuda_stream) if stream is not None else None
+        self._check(self._lib.gorio_link_probe(self._h, n_pulls, pages_in_flight, int(sequential), sp, ctypes.byref(gbs)))
+        return gbs.value
 
     def close(self):
         if self._h:

@@ -1,5 +1,5 @@
-// Query life cycle and the persistent kernel: page copies, the host poller, ticket hand-out,
-// the worker loop.
+// Query life cycle and the persistent kernel: page copies, the host poller, the poster, the puller
+// warps, ticket hand-out, the worker loop.
 // Part of the persistent search kernel; included by search_kernels.cu in this order.
 #pragma once
 #include "../gorio_internal.h"
@@ -63,6 +63,7 @@ __device__ void copy_page(const Ctx &c, u32 idx, u32 lane);
 template <bool PQ> __device__ void resident_worker(const Ctx &c, u32 lane, u32 *lut, u32 *ws);
 __host__ __device__ inline u32 resident_warp_words(u32 WR);
 __device__ bool warp_ticket(int *count, u32 *head, u32 &idx, u32 lane);
+__device__ void puller(const Ctx &c, u32 lane);
 
 // One unit of the work that keeps pages moving, in priority order: execute a copy the proxy
 // has admitted, consume a page the proxy has published (or a handed-off waiter chain), give
@@ -70,7 +71,7 @@ __device__ bool warp_ticket(int *count, u32 *head, u32 &idx, u32 lane);
 template <bool PQ>
 __device__ __noinline__ u32 service_step(const Ctx &c, u32 lane) {
   u32 v;
-  if (warp_ticket(&c.ctl->counts[0], &c.cs->copy_head, v, lane)) {    // the outstanding window waits on these
+  if (!c.pullers && warp_ticket(&c.ctl->counts[0], &c.cs->copy_head, v, lane)) {    // the outstanding window waits on these
     copy_page(c, v, lane);
     return 1;
   }
@@ -198,8 +199,9 @@ __device__ void run_query(const Ctx &c, u32 qs, u32 lane, u32 *lut, u32 &lut_qid
 
 // Execute the copy of admitted request idx (the proxy admits requests in ring order and
 // publishes how many; the request itself is read from the device copy of the ring): pull
-// the 4 KB page from the pinned store into its cache slot.  Any worker warp does this, ahead
-// of all other work; only the page bytes cross the host link on this path.  The host is told
+// the 4 KB page from the pinned store into its cache slot.  A puller warp does this (or, in the
+// shared scheme, any worker warp, ahead of all other work); only the page bytes cross the host link
+// on this path.  The host is told
 // as soon as the page's bytes have arrived on the GPU (they are in registers), so that no
 // fence sits inside the proxy's outstanding window; the stores into the slot are then
 // released to the consumers of the arrival through the slot's `filled` generation.
@@ -276,7 +278,9 @@ __device__ void census(const Ctx &c, u32 lane) {
 // every descriptor, so all the host has to say is two counters: how many requests are
 // admitted (their pages may be copied now) and how many completions are published (their
 // pages have "arrived").  One 16-byte read per iteration fetches both and the abort word;
-// the poller turns the deltas into tickets that worker warps take with fetch-and-add.
+// the poller passes the admitted count on to the puller warps (a word they wait on) and turns
+// new completions into tickets that worker warps take with fetch-and-add (in the shared scheme
+// admissions become tickets too).
 //
 // A control read is a PCIe read like any other: its completion queues behind the page data
 // already requested, so under load it takes about 6 us instead of 1.4 (46,000 reads in a 287 ms
@@ -294,7 +298,10 @@ __device__ void poller(const Ctx &c, u32 lane) {
       const uint4 h = ld_sys_v4(c.host_ctl);       // ~6 us under load; the stop flag's load rides along
       stop = ld_u32(&c.ctl->stop);
       pub = h.x; abort_req = h.y; adm = h.z;
-      if (adm != seen_adm) atomicAdd(&c.ctl->counts[0], (int)(adm - seen_adm));
+      if (adm != seen_adm) {
+        if (c.pullers) st_u32(&c.ctl->adm_seen, adm);        // the puller warps wait on this word
+        else atomicAdd(&c.ctl->counts[0], (int)(adm - seen_adm));
+      }
       if (pub != seen_pub) atomicAdd(&c.ctl->counts[1], (int)(pub - seen_pub));
       if (adm == seen_adm && pub == seen_pub) __nanosleep(100);
       seen_adm = adm; seen_pub = pub;
@@ -332,6 +339,40 @@ __device__ void poster(const Ctx &c, u32 lane) {
   }
 }
 
+// Puller warps (the last warp of every block when pages are pulled by the SMs): each claims the
+// next request index in ring order ahead of time, waits until the poller has seen that request
+// admitted, and pulls its page.  Pulls are thus issued in admission order, by warps that are
+// doing nothing else, the moment the admission is known on the GPU -- the proxy publishes
+// completions in that same order, so a pull that starts late holds up every request behind it.
+__device__ void puller(const Ctx &c, u32 lane) {
+  const u64 t0 = globaltimer();
+  u64 t_cpy = 0;
+  for (;;) {
+    u32 idx = 0;
+    if (lane == 0) idx = atomicAdd(&c.cs->copy_head, 1u);
+    idx = __shfl_sync(0xffffffffu, idx, 0);
+    bool go = false;
+    for (u32 it = 0;; ++it) {
+      u32 st = 0;
+      if (lane == 0) {
+        if ((int)(ld_u32(&c.ctl->adm_seen) - idx) > 0) st = 1u;
+        else if (ld_u32(&c.ctl->stop)) st = 2u;
+        else if ((it & 1023u) == 1023u && globaltimer() - t0 > c.timeout_ns) st = 3u;
+      }
+      st = __shfl_sync(0xffffffffu, st, 0);
+      if (st == 1u) { go = true; break; }
+      if (st == 3u && lane == 0) raise(c, 5, 0xB6, idx);
+      if (st) break;
+      __nanosleep(it < 16u ? 50u : 400u);
+    }
+    if (!go) break;
+    const u64 t1 = globaltimer();
+    copy_page(c, idx, lane);
+    t_cpy += globaltimer() - t1;
+  }
+  if (lane == 0) atomicAdd((unsigned long long *)&c.ctl->stats[S_T_CPY], t_cpy);
+}
+
 // Take one ticket from a (count, head) pair released by the poller; lane 0 only.
 __device__ __forceinline__ bool take_ticket(int *count, u32 *head, u32 &idx) {
   if ((int)ld_u32((const u32 *)count) <= 0) return false;
@@ -357,6 +398,7 @@ __global__ void __launch_bounds__(MAXT, 1) search_kernel(const Ctx c) {
   const u32 lane = lane_id(), warp = threadIdx.x >> 5;
   if (blockIdx.x == 0 && warp == 0) { poller(c, lane); return; }
   if (blockIdx.x == 0 && warp == 1 && !c.identity) { poster(c, lane); return; }     // (nothing is ever posted when the whole index is resident)
+  if (c.pullers && warp == (blockDim.x >> 5) - 1u) { puller(c, lane); return; }
   u32 *lut = PQ ? smem_lut + (u64)warp * c.pq_m * kPqLutWords : nullptr;
   // this warp's candidate area (WR keys and 16 frontier ids), behind the PQ tables
   u32 *ws = smem_lut + (PQ ? (u64)(blockDim.x >> 5) * c.pq_m * kPqLutWords : 0) + (u64)warp * resident_warp_words(c.WR);

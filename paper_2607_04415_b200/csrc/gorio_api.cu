@@ -493,6 +493,10 @@ void fill_ctx(gorio_index *ix, const void *queries_dev, u32 nq, u32 K, u32 L, u3
   c.dma_fill = ix->cfg.copy_mode == GORIO_COPY_ENGINE ? 1u : 0u;
   c.identity = whole_index_resident(ix) ? 1u : 0u;
   c.resident_fast = resident_fast_path(ix, K, W) ? 1u : 0u;
+  // who pulls pages (SM pull): one dedicated warp per block, in ring order -- unless nothing is ever
+  // pulled (whole index resident, copy-engine fills), the unit is a record (request rates beyond
+  // what one warp per SM carries), or the caller asks for the shared scheme
+  c.pullers = (!c.dma_fill && !c.identity && !c.record_mode && !ix->tune.shared_pull) ? 1u : 0u;
 }
 
 // Launch geometry of the persistent kernel: blocks and warps per block.  Needs only the index, the
@@ -825,6 +829,37 @@ int gorio_stats(gorio_index *ix, gorio_stats_t *out) {
   out->warp_ns_arrivals = h.stats[S_T_ARR]; out->warp_ns_queries = h.stats[S_T_RUN]; out->warp_ns_idle = h.stats[S_T_IDLE];
   out->arrivals_consumed = h.stats[S_N_ARR]; out->warp_ns_copies = h.stats[S_T_CPY]; out->stash_hits = h.stats[S_STASH];
   out->fetched_bytes = ix->host_fetched_bytes;
+  return GORIO_OK;
+}
+
+int gorio_link_probe(gorio_index *ix, uint32_t n_pulls, uint32_t pages_in_flight, int sequential, void *cuda_stream,
+                     double *gbs_out) {
+  if (!ix || !gbs_out) return GORIO_ERR_INVALID_ARG;
+  std::lock_guard<std::recursive_mutex> api_lock(ix->api_mu);
+  if (n_pulls == 0 || pages_in_flight == 0 || pages_in_flight > 16384u)
+    return fail(ix, GORIO_ERR_INVALID_ARG, "link_probe: need n_pulls >= 1 and 1 <= pages_in_flight <= 16384");
+  CK(cudaSetDevice(ix->dev));
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  const u32 warps = (pages_in_flight + 3u) / 4u * 4u;        // whole blocks of four warps
+  u8 *scratch = nullptr;
+  u32 *words = nullptr;                                      // [0] next pull, [1] checksum sink
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  float ms = 0.f;
+  cudaError_t e = cudaMalloc(&scratch, (size_t)warps * kPageBytes);
+  if (e == cudaSuccess) e = cudaMalloc(&words, 8);
+  if (e == cudaSuccess) e = cudaEventCreate(&e0);
+  if (e == cudaSuccess) e = cudaEventCreate(&e1);
+  if (e == cudaSuccess) e = cudaMemsetAsync(words, 0, 8, stream);
+  if (e == cudaSuccess) e = cudaEventRecord(e0, stream);
+  if (e == cudaSuccess) e = launch_link_probe(ix->pages_dev, ix->n_pages, n_pulls, warps, sequential ? 1u : 0u, scratch, words, words + 1, stream);
+  if (e == cudaSuccess) e = cudaEventRecord(e1, stream);
+  if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+  if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  cudaFree(scratch); cudaFree(words);
+  if (e != cudaSuccess) return cuda_fail(ix, e, "link_probe");
+  *gbs_out = ms > 0.f ? (double)n_pulls * kPageBytes / ((double)ms * 1e6) : 0.0;
   return GORIO_OK;
 }
 

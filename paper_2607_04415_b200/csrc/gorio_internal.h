@@ -66,6 +66,7 @@ struct Ctl {
   u32 next_query;  // next query id to admit when a slot frees
   u32 done;        // queries finished
   u32 ring_head;   // request descriptors posted
+  u32 adm_seen;    // admitted-request count the poller last read from the host (puller warps wait on it)
   u32 q_heads[16]; // queue head/tail words: arr(0,1) run(3,4) want(6,7)
   u32 dbg[8];      // detail of the first error
   u32 census[16];  // debug snapshot (see census())
@@ -137,6 +138,7 @@ struct Ctx {
   u64 census_ns;   // debug: take a state census this long after the kernel started (0 = never)
   u32 max_iters;
   u32 idle_ns;       // longest sleep of an idle warp between looks at the work counters
+  u32 pullers;       // 1: the last warp of every block only pulls pages, in ring order; worker warps pull none
   u32 max_in_flight; // cap on posted-but-not-arrived requests
   u32 vec128;      // 1: vectors are whole 16-byte chunks (<= 24) and query rows are 16-byte aligned
   u32 blocking;    // 1: a warp waits in place for its query's pages instead of yielding
@@ -156,5 +158,7 @@ cudaError_t launch_search(const Ctx &c, u32 blocks, u32 warps_per_block, cudaStr
 cudaError_t search_occupancy(const Ctx &c, u32 warps_per_block, int *blocks_per_sm);
 size_t search_smem_per_warp(const Ctx &c);
 cudaError_t launch_cache_reset(const Ctx &c, u32 preloaded_pages, cudaStream_t s);
+cudaError_t launch_link_probe(const u8 *host_pages, u32 n_pages, u32 n_pulls, u32 warps, u32 sequential, u8 *scratch,
+                              u32 *next, u32 *sink, cudaStream_t s);
 
 }  // namespace gorio

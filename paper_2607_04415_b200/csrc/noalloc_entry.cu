@@ -151,6 +151,7 @@ extern "C" int gorio_search_resident_noalloc(const gorio_index_desc *d, const vo
   c.resident_fast = 1;      // ... so every query runs start to end on the warp that takes it
   c.max_in_flight = 1u << 30;
   c.idle_ns = 8000;
+  c.pullers = 0;
   c.vec128 = (c.vec_bytes % 16 == 0 && c.vec_bytes <= 384 && ((uintptr_t)queries_dev & 15) == 0 &&
               ((uintptr_t)pages_dev & 15) == 0) ? 1u : 0u;
 

@@ -15,6 +15,9 @@
 // consume it now; if the page is in flight register as a waiter; if it is absent claim a
 // slot (clock eviction), post a request descriptor (the poster warp forwards it to the
 // host-visible ring) and register.
+// Requests the host proxy has admitted are pulled from the pinned store by the puller warps (the
+// last warp of every block), in ring order; the proxy publishes each completion once the page's
+// bytes are on the GPU and the injected latency has passed.
 // A page that arrives is consumed for every registered waiter by whichever warp picks the
 // arrival up, using only the waiter's query vector, so no page stays pinned for a query.
 // The last item consumed of a batch pushes the query back onto the runnable queue.
@@ -52,7 +55,7 @@ __global__ void init_kernel(const Ctx c) {
     for (int i = 0; i < 8; ++i) ctl->dbg[i] = 0;
     *c.run.tail = c.n_qslots;
     *c.run.count = (int)c.n_qslots;
-    ctl->counts[0] = 0; ctl->counts[1] = 0; c.cs->copy_head = 0; c.cs->comp_head = 0; c.cs->in_flight = 0;
+    ctl->counts[0] = 0; ctl->counts[1] = 0; c.cs->copy_head = 0; c.cs->comp_head = 0; c.cs->in_flight = 0; ctl->adm_seen = 0;
   }
 }
 
@@ -72,6 +75,42 @@ __global__ void cache_reset_kernel(const Ctx c, u32 preloaded) {
 // ------------------------------------------------------------------------------------------
 // launchers
 // ------------------------------------------------------------------------------------------
+// Link probe: what the host link delivers to the access pattern of copy_page and nothing else.
+// Every warp pulls whole 4 KB pages of the pinned store into a 4 KB area of its own in HBM, one
+// page at a time with all of the page's loads in flight (exactly copy_page's loads), pull i going
+// to page hash(i) mod n_pages (or page i mod n_pages when `sequential`).  The number of warps is
+// the number of pages in flight.  No cache, no proxy, no queries.
+__global__ void __launch_bounds__(128) link_probe_kernel(const u8 *host_pages, u32 n_pages, u32 n_pulls, u32 sequential,
+                                                         u8 *scratch, u32 *next, u32 *sink) {
+  const u32 lane = threadIdx.x & 31u;
+  const u32 warp = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  uint4 *dst = (uint4 *)(scratch + (u64)warp * kPageBytes);
+  u32 acc = 0;
+  for (;;) {
+    u32 i = 0;
+    if (lane == 0) i = atomicAdd(next, 1u);
+    i = __shfl_sync(0xffffffffu, i, 0);
+    if (i >= n_pulls) break;
+    const u32 page = (sequential ? i : hash32(i)) % n_pages;
+    const uint4 *src = (const uint4 *)(host_pages + (u64)page * kPageBytes);
+    uint4 v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v[k] = __ldcs(src + k * 32 + lane);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) acc ^= v[k].x ^ v[k].y ^ v[k].z ^ v[k].w;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) __stcg(dst + k * 32 + lane, v[k]);
+  }
+  acc = __reduce_xor_sync(0xffffffffu, acc);
+  if (lane == 0) atomicXor(sink, acc);
+}
+
+cudaError_t launch_link_probe(const u8 *host_pages, u32 n_pages, u32 n_pulls, u32 warps, u32 sequential, u8 *scratch,
+                              u32 *next, u32 *sink, cudaStream_t s) {
+  link_probe_kernel<<<(warps + 3) / 4, 128, 0, s>>>(host_pages, n_pages, n_pulls, sequential, scratch, next, sink);
+  return cudaGetLastError();
+}
+
 // With lazy module loading the first launch of a kernel may need a context-wide
 // synchronisation; querying the attributes loads all code at open time instead, so that no
 // launch ever has to wait behind a resident persistent kernel.
@@ -82,6 +121,7 @@ cudaError_t preload_kernels() {
   if ((e = cudaFuncGetAttributes(&a, search_kernel<false, 768>)) != cudaSuccess) return e;
   if ((e = cudaFuncGetAttributes(&a, search_kernel<true, 384>)) != cudaSuccess) return e;
   if ((e = cudaFuncGetAttributes(&a, init_kernel)) != cudaSuccess) return e;
+  if ((e = cudaFuncGetAttributes(&a, link_probe_kernel)) != cudaSuccess) return e;
   return cudaFuncGetAttributes(&a, cache_reset_kernel);
 }
 

@@ -171,6 +171,41 @@ def test_copy_engine_dedupe_proof_and_config3_shape(gorio, cfg1):
     _assert_exact(got3, ref3)
 
 
+@pytest.mark.parametrize("shared,warps,pq", [(0, 0, False), (1, 0, False), (0, 2, False), (0, 3, False), (0, 0, True), (1, 0, True)])
+def test_puller_warps_and_shared_pull_both_match_oracle(gorio, shared, warps, pq):
+    """Who pulls admitted pages: by default the last warp of every block does nothing else and
+    pulls in ring order; tuning.shared_pull hands the pulls back to the worker warps.  Same
+    results either way, also with the fewest warps per block (2: block 0 is poller and poster only,
+    every other block one worker and one puller) and with PQ navigation."""
+    w = make_config(3, scale=0.02, nq=300, with_gt=False)              # 10 nodes per page, R = 64
+    if pq:
+        w.pq_centroids, w.pq_codes = train_pq(w.data, m=32, sample=4096, iters=3)
+    ref = OracleIndex.from_workload(w, use_pq=pq).search(w.queries, w.K, w.L, w.W, threads=4)
+    got = _gpu_search(gorio, w, w.cache_pages, use_pq=pq, remote_latency_ns=5000, max_outstanding=64,
+                      tuning=dict(shared_pull=shared, warps_per_block=warps))
+    _assert_exact(got, ref)
+    st = got["stats"]
+    assert st["pages_fetched"] > 0 and st["max_outstanding_seen"] <= 64 and st["warp_ns_copies"] > 0
+
+
+def test_link_probe_reports_a_plausible_rate(gorio, cfg1):
+    """gorio_link_probe pulls pages of the pinned store with the loads of a page fill and nothing
+    else; it must return a positive rate below the link's nominal 64 GB/s and reject bad arguments."""
+    w, _ = cfg1
+    ix = gorio.Index.from_workload(w)
+    try:
+        ix.cache_config(64)
+        for seq in (False, True):
+            gbs = ix.link_probe(20000, 64, sequential=seq)
+            assert 1.0 < gbs < 64.0
+        for bad in ((0, 64), (100, 0), (100, 20000)):
+            with pytest.raises(gorio.GorioError) as e:
+                ix.link_probe(*bad)
+            assert e.value.status == 1
+    finally:
+        ix.close()
+
+
 @pytest.mark.parametrize("K,L,W", [(1, 1, 1), (10, 10, 1), (64, 64, 4), (10, 200, 8), (100, 256, 16), (5, 33, 3)])
 def test_parameter_edges(gorio, cfg1, K, L, W):
     w, _ = cfg1
@@ -664,7 +699,7 @@ def test_randomized_configurations_match_oracle(gorio, seed):
     cap = int(rng.integers(16, max(17, w.n_pages + 1)))
     tuning = dict(warps_per_block=int(rng.integers(2, 17)), max_inflight=int(rng.choice([0, 8, 64])),
                   stash_entries=int(rng.choice([0, 1, 64, 256])), blocking=int(rng.integers(0, 2)),
-                  request_backlog=int(rng.choice([0, 1, 16, 4096])))
+                  request_backlog=int(rng.choice([0, 1, 16, 4096])), shared_pull=int(rng.integers(0, 3) == 0))
     preload, lat, depth = bool(rng.integers(0, 4) == 0), int(rng.choice([0, 2000, 20000])), int(rng.choice([1, 8, 256]))
     copy_engine, gran = bool(rng.integers(0, 4) == 0), str(rng.choice(["page", "page", "record"]))
     got = _gpu_search(gorio, w, cap, K=K, L=L, W=W, tuning=tuning, preload=preload and gran == "page",
