@@ -203,7 +203,9 @@ typedef struct {
   uint64_t proxy_service_ns, proxy_iters, proxy_ack_wait_iters, proxy_window_full_iters;
   uint64_t proxy_ring_empty_iters, proxy_outstanding_sum;
   /* where the worker warps' time went, ns summed over warps: serving arrived pages,
-     running query phases, idle; the number of arrival-queue items consumed; ns executing copy commands */
+     running query phases, idle; the number of arrival-queue items consumed; ns spent pulling
+     pages (by the puller warps, whose waiting for the next admission is not counted anywhere, or in
+     the shared scheme by the worker warps) */
   uint64_t warp_ns_arrivals, warp_ns_queries, warp_ns_idle, arrivals_consumed;
   uint64_t warp_ns_copies, stash_hits;   /* expansions served from the adjacency stash */
   uint64_t fetched_bytes;
