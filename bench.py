@@ -217,6 +217,8 @@ def main():
     ap.add_argument("--warps", type=int, default=0, help="warps per block of the persistent kernel (0 = the library's choice)")
     ap.add_argument("--visited-capacity", type=int, default=0,
                     help="entries of the per-query visited set (0 = the library's default; a bitmap is used when it is no larger)")
+    ap.add_argument("--request-backlog", type=int, default=0,
+                    help="most requests posted and not yet arrived (0 = the library's default, 4 x the window up to 1024)")
     ap.add_argument("--shared-pull", action="store_true",
                     help="ablation: worker warps pull admitted pages between their other work (no dedicated puller warps)")
     ap.add_argument("--no-fast-path", action="store_true", help="whole index resident: use the general path anyway")
@@ -288,9 +290,10 @@ def main():
     lat_ns, max_out = int(w.latency_us * 1000), w.max_outstanding
     use_pq = args.config == 4
     ix = g.Index.from_workload(w, device=local, use_pq=use_pq)
-    if args.blocking or args.warps or args.no_fast_path or args.shared_pull or args.visited_capacity:
+    if args.blocking or args.warps or args.no_fast_path or args.shared_pull or args.visited_capacity or args.request_backlog:
         ix.set_tuning(blocking=int(args.blocking), warps_per_block=args.warps, no_fast_path=int(args.no_fast_path),
-                      visited_capacity=args.visited_capacity, shared_pull=int(args.shared_pull))
+                      visited_capacity=args.visited_capacity, shared_pull=int(args.shared_pull),
+                      request_backlog=args.request_backlog)
     q_dev = torch.as_tensor(my_q).to(dev)
     q_pin = torch.as_tensor(my_q).pin_memory()
     outs_pin = dict(ids=torch.empty((my_nq, w.K), dtype=torch.int32).pin_memory(),
