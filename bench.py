@@ -257,6 +257,10 @@ def main():
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if world > 1:
+        # one rank per GPU: keep this rank's page store, proxy thread and polled words on the GPU's socket
+        from paper_2607_04415_b200.shard import bind_to_gpu_cpus
+        pr = torch.cuda.get_device_properties(local)
+        bind_to_gpu_cpus(f"{pr.pci_domain_id:04x}:{pr.pci_bus_id:02x}:{pr.pci_device_id:02x}.0")
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
         if dist.get_world_size() != args.gpus:

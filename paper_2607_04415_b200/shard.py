@@ -49,3 +49,35 @@ def spawn_ranks(n_ranks: int, script: str, argv, env=None, timeout=None) -> int:
     for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE"):      # the launcher sets these for its children
         e.pop(k, None)
     return subprocess.run(cmd, env=e, timeout=timeout).returncode
+
+
+def parse_cpulist(text: str):
+    """'0-3,8,10-11' -> {0, 1, 2, 3, 8, 10, 11} (the format of sysfs cpulist files)."""
+    cpus = set()
+    for part in text.strip().split(","):
+        if not part:
+            continue
+        lo, _, hi = part.partition("-")
+        cpus.update(range(int(lo), int(hi or lo) + 1))
+    return cpus
+
+
+def bind_to_gpu_cpus(pci_bus: str, sysfs_root: str = "/sys") -> bool:
+    """Restrict this process to the CPUs next to a GPU (sysfs `local_cpulist` of its PCI device), so
+    that the page store a rank allocates and pins afterwards, its proxy thread and the words that
+    thread polls sit on the GPU's own socket: with one rank per GPU on a two-socket host, a page
+    store on the far socket makes every page pull cross the socket interconnect.  Best effort: it
+    does nothing (and returns False) when the file is missing, names no CPU this process may use,
+    or names all of them.  `pci_bus` is 'dddd:bb:dd.f', lower case."""
+    import os
+    try:
+        with open(os.path.join(sysfs_root, "bus/pci/devices", pci_bus, "local_cpulist")) as fh:
+            local = parse_cpulist(fh.read())
+        allowed = os.sched_getaffinity(0)
+        want = local & allowed
+        if not want or want == allowed:
+            return False
+        os.sched_setaffinity(0, want)
+        return True
+    except (OSError, ValueError):
+        return False

@@ -219,3 +219,29 @@ def test_bench_reference_arm_prints_the_contract_line_on_cpu():
     assert line["impl"] == "reference" and line["value"] > 0 and line["vs_baseline"] is None
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
+
+
+def test_bind_to_gpu_cpus_follows_sysfs_and_is_a_no_op_when_it_cannot_help(tmp_path):
+    """The rank-to-socket binding reads the PCI device's local_cpulist: it narrows the affinity to the
+    CPUs named there that this process may use, and leaves it alone when the file is missing, names
+    none of them, or names all of them."""
+    import os
+    from paper_2607_04415_b200.shard import bind_to_gpu_cpus, parse_cpulist
+    assert parse_cpulist("0-3,8,10-11\n") == {0, 1, 2, 3, 8, 10, 11}
+    allowed = os.sched_getaffinity(0)
+    dev = tmp_path / "bus/pci/devices/0000:aa:00.0"
+    dev.mkdir(parents=True)
+    try:
+        assert not bind_to_gpu_cpus("0000:bb:00.0", str(tmp_path))                 # no such device
+        (dev / "local_cpulist").write_text(",".join(str(c) for c in sorted(allowed)) + "\n")
+        assert not bind_to_gpu_cpus("0000:aa:00.0", str(tmp_path))                 # names every allowed CPU
+        (dev / "local_cpulist").write_text(str(max(allowed) + 1000) + "\n")
+        assert not bind_to_gpu_cpus("0000:aa:00.0", str(tmp_path))                 # names none of them
+        assert os.sched_getaffinity(0) == allowed
+        if len(allowed) > 1:
+            one = min(allowed)
+            (dev / "local_cpulist").write_text(f"{one}\n")
+            assert bind_to_gpu_cpus("0000:aa:00.0", str(tmp_path))
+            assert os.sched_getaffinity(0) == {one}
+    finally:
+        os.sched_setaffinity(0, allowed)
