@@ -398,7 +398,7 @@ __global__ void __launch_bounds__(MAXT, 1) search_kernel(const Ctx c) {
   const u32 lane = lane_id(), warp = threadIdx.x >> 5;
   if (blockIdx.x == 0 && warp == 0) { poller(c, lane); return; }
   if (blockIdx.x == 0 && warp == 1 && !c.identity) { poster(c, lane); return; }     // (nothing is ever posted when the whole index is resident)
-  if (c.pullers && warp == (blockDim.x >> 5) - 1u) { puller(c, lane); return; }
+  if (blockIdx.x < c.pullers && warp == (blockDim.x >> 5) - 1u) { puller(c, lane); return; }
   u32 *lut = PQ ? smem_lut + (u64)warp * c.pq_m * kPqLutWords : nullptr;
   // this warp's candidate area (WR keys and 16 frontier ids), behind the PQ tables
   u32 *ws = smem_lut + (PQ ? (u64)(blockDim.x >> 5) * c.pq_m * kPqLutWords : 0) + (u64)warp * resident_warp_words(c.WR);

@@ -496,7 +496,7 @@ void fill_ctx(gorio_index *ix, const void *queries_dev, u32 nq, u32 K, u32 L, u3
   // who pulls pages (SM pull): one dedicated warp per block, in ring order -- unless nothing is ever
   // pulled (whole index resident, copy-engine fills), the unit is a record (request rates beyond
   // what one warp per SM carries), or the caller asks for the shared scheme
-  c.pullers = (!c.dma_fill && !c.identity && !c.record_mode && !ix->tune.shared_pull) ? 1u : 0u;
+  c.pullers = (!c.dma_fill && !c.identity && !c.record_mode && !ix->tune.shared_pull) ? (u32)ix->n_sms : 0u;     // one per SM, also with two blocks per SM
 }
 
 // Launch geometry of the persistent kernel: blocks and warps per block.  Needs only the index, the

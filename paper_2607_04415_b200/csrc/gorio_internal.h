@@ -138,7 +138,8 @@ struct Ctx {
   u64 census_ns;   // debug: take a state census this long after the kernel started (0 = never)
   u32 max_iters;
   u32 idle_ns;       // longest sleep of an idle warp between looks at the work counters
-  u32 pullers;       // 1: the last warp of every block only pulls pages, in ring order; worker warps pull none
+  u32 pullers;       // blocks 0 .. pullers-1 (one per SM) give their last warp to pulling pages, in ring order;
+                     // worker warps then pull none.  0: the shared scheme (worker warps take the pulls)
   u32 max_in_flight; // cap on posted-but-not-arrived requests
   u32 vec128;      // 1: vectors are whole 16-byte chunks (<= 24) and query rows are 16-byte aligned
   u32 blocking;    // 1: a warp waits in place for its query's pages instead of yielding

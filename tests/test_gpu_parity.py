@@ -171,18 +171,20 @@ def test_copy_engine_dedupe_proof_and_config3_shape(gorio, cfg1):
     _assert_exact(got3, ref3)
 
 
-@pytest.mark.parametrize("shared,warps,pq", [(0, 0, False), (1, 0, False), (0, 2, False), (0, 3, False), (0, 0, True), (1, 0, True)])
-def test_puller_warps_and_shared_pull_both_match_oracle(gorio, shared, warps, pq):
+@pytest.mark.parametrize("shared,warps,pq,bps", [(0, 0, False, 0), (1, 0, False, 0), (0, 2, False, 0), (0, 3, False, 0),
+                                                 (0, 0, True, 0), (1, 0, True, 0), (0, 4, False, 2)])
+def test_puller_warps_and_shared_pull_both_match_oracle(gorio, shared, warps, pq, bps):
     """Who pulls admitted pages: by default the last warp of every block does nothing else and
     pulls in ring order; tuning.shared_pull hands the pulls back to the worker warps.  Same
     results either way, also with the fewest warps per block (2: block 0 is poller and poster only,
-    every other block one worker and one puller) and with PQ navigation."""
+    every other block one worker and one puller), with two blocks per SM (still one puller per SM's
+    worth of blocks) and with PQ navigation."""
     w = make_config(3, scale=0.02, nq=300, with_gt=False)              # 10 nodes per page, R = 64
     if pq:
         w.pq_centroids, w.pq_codes = train_pq(w.data, m=32, sample=4096, iters=3)
     ref = OracleIndex.from_workload(w, use_pq=pq).search(w.queries, w.K, w.L, w.W, threads=4)
     got = _gpu_search(gorio, w, w.cache_pages, use_pq=pq, remote_latency_ns=5000, max_outstanding=64,
-                      tuning=dict(shared_pull=shared, warps_per_block=warps))
+                      tuning=dict(shared_pull=shared, warps_per_block=warps, blocks_per_sm=bps))
     _assert_exact(got, ref)
     st = got["stats"]
     assert st["pages_fetched"] > 0 and st["max_outstanding_seen"] <= 64 and st["warp_ns_copies"] > 0
