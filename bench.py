@@ -494,7 +494,8 @@ def main():
             "pages_fetched": fetched, "fetched_bytes": fetched_bytes, "algorithmic_hbm_bytes": b_hbm,
             "hbm_achieved_gbs": b_hbm / (ms * 1e-3) / 1e9, "hbm_peak_gbs": pk["hbm_gbs"],
             "host_link_bulk_copy_gbs": h2d, "host_link_sm_page_pull_gbs": sm_pull_gbs,
-            "fetched_gbs": fetched_bytes / (ms * 1e-3) / 1e9}
+            "fetched_gbs": fetched_bytes / (ms * 1e-3) / 1e9,
+            "fetched_over_sm_page_pull": fetched_bytes / (ms * 1e-3) / 1e9 / sm_pull_gbs if sm_pull_gbs > 0 else None}
     if default_workload:
         # DRAM bytes of one search_kernel launch from a single-pass ncu capture of this command, valid
         # only for the device code it was captured on
